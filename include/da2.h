@@ -1,0 +1,135 @@
+/*
+ * da2 -- DraftAttention2 attention hot path for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * Low-resolution-guided block selection with mixed-precision block-sparse attention:
+ *   da2_plan          host only: spatial tiling, quotas, workspace layout      (Sec. 3.3, App. C.1/C.2)
+ *   da2_prepare       device: pool -> draft map -> rank/tag/lists -> operand quantisation
+ *                                                                    (Eq. v2-descriptors, Def. 3.1, Alg. 1, App. C.3)
+ *   da2_attention_fwd device: one phased kernel, NVFP4 -> INT8/E4M3 -> BF16 segments sharing one
+ *                     online-softmax state and one output accumulator          (Sec. 3.3, App. C.4)
+ *
+ * Conventions
+ *   - q, k, v, out: DEVICE pointers, contiguous bf16 [B, H, N, head_dim], N = T*Hg*Wg, raster token order
+ *     u = (t*Hg + y)*Wg + x, 16-byte aligned.  out must not alias the inputs.
+ *   - workspace: DEVICE pointer, 256-byte aligned, at least da2_plan_info().workspace_bytes long.  The caller owns
+ *     all device memory; the library allocates none and keeps no device state between calls.
+ *   - stream: a cudaStream_t passed as void* (NULL = default stream).  da2_prepare and da2_attention_fwd only
+ *     enqueue work and never synchronise.
+ *   - Errors are return codes.  Argument errors are detected before any launch.  A device-side bounded wait that
+ *     gives up records a code in the workspace status word; da2_device_status reports it.
+ *   - The plan is host memory owned by the library until da2_plan_destroy; it is immutable and may be reused for
+ *     any number of calls with the same shapes and budgets (the partition is reused across layers and steps).
+ */
+#ifndef DA2_H_
+#define DA2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DA2_OK = 0,
+  DA2_ERR_INVALID_ARG = 1,
+  DA2_ERR_UNSUPPORTED = 2,
+  DA2_ERR_WORKSPACE_TOO_SMALL = 3,
+  DA2_ERR_CUDA = 4,
+  DA2_ERR_TIMEOUT = 5,
+  DA2_ERR_INTERNAL = 6
+} da2_status_t;
+
+/* Scope of the shared ranking (Alg. 1).  ROW: every query-block row keeps the same number of key blocks per
+ * precision (the benchmark configurations).  HEAD: one ranking over all R*R region pairs of a head, as printed in
+ * Alg. 1, so rows may keep different numbers of blocks, possibly none. */
+typedef enum { DA2_RANK_ROW = 0, DA2_RANK_HEAD = 1 } da2_rank_scope_t;
+
+typedef struct {
+  int32_t B, H, T, Hg, Wg, head_dim; /* head_dim in {64, 128} */
+  int32_t tile_h, tile_w;            /* spatial tile of one block; only 8 x 8 is supported */
+  double frac16, frac8, frac4;       /* budgets as fractions of key blocks: bf16 / INT8+E4M3 / NVFP4; sum <= 1 */
+  float lambda;                      /* weight of the max-pooled draft branch in [0,1] (Def. 3.1) */
+  float softmax_scale;               /* <= 0 selects 1/sqrt(head_dim) */
+  int32_t rank_scope;                /* da2_rank_scope_t */
+  int32_t reserved;                  /* must be 0 */
+  const float *g_q, *g_k, *g_v;      /* optional HOST arrays [B*H]: NVFP4 per-tensor scales (App. C.3, g_X); NULL =
+                                        derived per head as amax/2688.  Copied into the plan. */
+} da2_config_t;
+
+typedef struct da2_plan da2_plan_t;
+
+/* Everything a caller (or a parity harness) needs to size and read the workspace.  Offsets are bytes from the
+ * workspace base.  "tier" index: 0 = NVFP4 (4-bit), 1 = INT8/E4M3 (8-bit), 2 = BF16 (16-bit). */
+typedef struct {
+  int32_t B, H, T, Hg, Wg, head_dim, tile_h, tile_w;
+  int32_t nty, ntx, R_f, R, S;       /* tiles per frame, blocks per head, slots per block (64) */
+  int64_t N;
+  int32_t rank_scope;
+  int32_t tier_active[3];            /* 1 if the tier has a non-zero quota */
+  int64_t quota[3];                  /* (k4, k8, k16): per row (ROW scope) or per head (HEAD scope) */
+  int64_t ids_per_head;              /* uint16 entries of the id array belonging to one head */
+  float lambda, softmax_scale;
+  uint64_t workspace_bytes;
+  uint64_t off_status;               /* int32[64]: [0] status code, [1..] diagnostics */
+  uint64_t off_amax;                 /* uint32[BH][4]: fp32 bit patterns of max|Q|, max|K|, max|V| per head */
+  uint64_t off_vmax;                 /* uint32[BH][d]: fp32 bit patterns of max_v |V_vc| */
+  uint64_t off_gscale;               /* fp32[BH][4]: NVFP4 per-tensor scales g_Q, g_K, g_V */
+  uint64_t off_desc[4];              /* fp32[BH][R][d]: Qavg, Qmax, Kavg, Kmax */
+  uint64_t off_logits[2];            /* fp32[BH][R][R]: draft logits of the average / max branch (scratch) */
+  uint64_t off_map;                  /* fp32[BH][R][R]: draft map A (Def. 3.1) */
+  uint64_t off_counts;               /* int32[BH][R][4]: (n4, n8, n16, offset of the row's ids inside its head) */
+  uint64_t off_ids;                  /* uint16[BH][ids_per_head]: key-block ids, per row 4-bit | 8-bit | 16-bit
+                                        segments, ascending inside a segment */
+  uint64_t off_select;               /* scratch of the HEAD-scope selection */
+  uint64_t off_qrec[3];              /* per tier: Q operand records [BH][R][qrec_bytes] */
+  uint64_t off_kvrec[3];             /* per tier: K + V operand records [BH][R][kvrec_bytes] */
+  uint32_t qrec_bytes[3], kvrec_bytes[3];
+  uint64_t off_dq8, off_dk8;         /* fp32[BH][R]: INT8 block scales of Q and K */
+  uint64_t off_dv8;                  /* fp32[BH][d]: E4M3 per-channel scale of V */
+} da2_plan_info_t;
+
+/*
+ * Operand record layouts (what da2_prepare writes and da2_attention_fwd streams into shared memory unchanged).
+ * A "K-major image" of a [rows x kbytes] matrix stores 16-byte chunks: chunk (kc, r) at byte (kc*rows + r)*16,
+ * i.e. 8 x 16 B core matrices, row-group stride 128 B, K-chunk stride rows*16 B.
+ *   Q record, tier 2: image of bf16 [64 slots x d]                      (128*d/8 ... = 2*64*d bytes)
+ *             tier 1: image of int8 [64 x d]                            (64*d bytes)
+ *             tier 0: image of packed E2M1 [64 x d/2 bytes], then d/64 scale atoms of 512 B
+ *   KV record: K part exactly like the Q record of the tier, then the V part:
+ *             tier 2: image of bf16 V^T [d channels x 64 slots]
+ *             tier 1: image of E4M3 V^T [d x 64]
+ *             tier 0: image of packed E2M1 V^T [d x 32 bytes], then one 512 B scale atom
+ *   Packed E2M1: element 2i in the low nibble of byte i.  Scale atom (E4M3 codes, one per 16 elements along the
+ *   reduction dimension): byte (row%32)*16 + (row/32)*4 + group, rows >= 64 unused for Q/K.
+ *   Padding slots of ragged edge tiles hold zeros.
+ */
+
+/* Builds the plan.  Host only; no CUDA call.  cfg and *plan_out must be non-NULL. */
+da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out);
+
+/* Fills *info.  Host only. */
+da2_status_t da2_plan_info(const da2_plan_t *plan, da2_plan_info_t *info);
+
+/* Pool, draft map, ranking, lists and operand records for (q, k, v) into workspace.  Enqueues on stream. */
+da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
+                         size_t workspace_bytes, void *stream);
+
+/* Phased mixed-precision block-sparse attention.  workspace must have been filled by da2_prepare for the same
+ * q, k, v (ordering on the same stream is enough).  Rows whose list is empty give zeros (App. C.1). */
+da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                               const void *workspace, void *out, void *stream);
+
+/* Synchronises stream, reads the workspace status word; DA2_OK, DA2_ERR_TIMEOUT or DA2_ERR_INTERNAL. */
+da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, void *stream);
+
+/* Number of kernels the last da2_prepare / da2_attention_fwd call on this plan enqueued (for launch accounting). */
+int32_t da2_last_launch_count(const da2_plan_t *plan);
+
+void da2_plan_destroy(da2_plan_t *plan);
+const char *da2_status_string(da2_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DA2_H_ */

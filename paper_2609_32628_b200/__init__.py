@@ -1,0 +1,14 @@
+"""da2: DraftAttention2's attention hot path for NVIDIA B200, hand-written sm_100a CUDA behind a C ABI.
+
+This package is a thin ctypes binding over ``libda2.so`` (built in-tree from ``csrc/`` by ``build.py``).
+Every step of the path runs in the library's kernels; Python only marshals arguments.  There is no CPU
+fallback: importing works without a GPU (so the library can be built and its symbols checked), but any
+compute call requires the CUDA library and a device.
+"""
+from .binding import (Da2Error, Plan, PlanInfo, STATUS, load_library, da2_plan, da2_plan_info, da2_prepare,
+                      da2_attention_fwd, da2_device_status, da2_plan_destroy, da2_status_string,
+                      da2_last_launch_count, attention)
+
+__all__ = ["Da2Error", "Plan", "PlanInfo", "STATUS", "load_library", "da2_plan", "da2_plan_info", "da2_prepare",
+           "da2_attention_fwd", "da2_device_status", "da2_plan_destroy", "da2_status_string",
+           "da2_last_launch_count", "attention"]

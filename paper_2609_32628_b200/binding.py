@@ -1,0 +1,180 @@
+"""ctypes binding of the da2 C ABI (include/da2.h).  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libda2.so")
+_lib = None
+
+STATUS = {0: "DA2_OK", 1: "DA2_ERR_INVALID_ARG", 2: "DA2_ERR_UNSUPPORTED", 3: "DA2_ERR_WORKSPACE_TOO_SMALL",
+          4: "DA2_ERR_CUDA", 5: "DA2_ERR_TIMEOUT", 6: "DA2_ERR_INTERNAL"}
+DA2_RANK_ROW, DA2_RANK_HEAD = 0, 1
+
+
+class Da2Error(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)} ({da2_status_string(code)})")
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("Hg", ctypes.c_int32),
+                ("Wg", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("tile_h", ctypes.c_int32),
+                ("tile_w", ctypes.c_int32), ("frac16", ctypes.c_double), ("frac8", ctypes.c_double),
+                ("frac4", ctypes.c_double), ("lambda_", ctypes.c_float), ("softmax_scale", ctypes.c_float),
+                ("rank_scope", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("g_q", ctypes.POINTER(ctypes.c_float)), ("g_k", ctypes.POINTER(ctypes.c_float)),
+                ("g_v", ctypes.POINTER(ctypes.c_float))]
+
+
+class PlanInfo(ctypes.Structure):
+    """Mirror of da2_plan_info_t."""
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("Hg", ctypes.c_int32),
+                ("Wg", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("tile_h", ctypes.c_int32),
+                ("tile_w", ctypes.c_int32), ("nty", ctypes.c_int32), ("ntx", ctypes.c_int32),
+                ("R_f", ctypes.c_int32), ("R", ctypes.c_int32), ("S", ctypes.c_int32), ("N", ctypes.c_int64),
+                ("rank_scope", ctypes.c_int32), ("tier_active", ctypes.c_int32 * 3), ("quota", ctypes.c_int64 * 3),
+                ("ids_per_head", ctypes.c_int64), ("lambda_", ctypes.c_float), ("softmax_scale", ctypes.c_float),
+                ("workspace_bytes", ctypes.c_uint64), ("off_status", ctypes.c_uint64), ("off_amax", ctypes.c_uint64),
+                ("off_vmax", ctypes.c_uint64), ("off_gscale", ctypes.c_uint64), ("off_desc", ctypes.c_uint64 * 4),
+                ("off_logits", ctypes.c_uint64 * 2), ("off_map", ctypes.c_uint64), ("off_counts", ctypes.c_uint64),
+                ("off_ids", ctypes.c_uint64), ("off_select", ctypes.c_uint64), ("off_qrec", ctypes.c_uint64 * 3),
+                ("off_kvrec", ctypes.c_uint64 * 3), ("qrec_bytes", ctypes.c_uint32 * 3),
+                ("kvrec_bytes", ctypes.c_uint32 * 3), ("off_dq8", ctypes.c_uint64), ("off_dk8", ctypes.c_uint64),
+                ("off_dv8", ctypes.c_uint64)]
+
+
+def load_library():
+    """Loads libda2.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2609_32628_b200.build` "
+                               "(the da2 path has no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(_LIB_PATH)
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        lib.da2_plan.restype = ctypes.c_int
+        lib.da2_plan.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp)]
+        lib.da2_plan_info.restype = ctypes.c_int
+        lib.da2_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+        lib.da2_prepare.restype = ctypes.c_int
+        lib.da2_prepare.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+        lib.da2_attention_fwd.restype = ctypes.c_int
+        lib.da2_attention_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        lib.da2_device_status.restype = ctypes.c_int
+        lib.da2_device_status.argtypes = [vp, vp, vp]
+        lib.da2_last_launch_count.restype = ctypes.c_int32
+        lib.da2_last_launch_count.argtypes = [vp]
+        lib.da2_plan_destroy.restype = None
+        lib.da2_plan_destroy.argtypes = [vp]
+        lib.da2_status_string.restype = ctypes.c_char_p
+        lib.da2_status_string.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def da2_status_string(code: int) -> str:
+    return load_library().da2_status_string(int(code)).decode()
+
+
+class Plan:
+    """Owns a da2_plan_t handle."""
+
+    def __init__(self, handle: int):
+        self.handle = ctypes.c_void_p(handle)
+        self.info = da2_plan_info(self)
+
+    def close(self):
+        if self.handle:
+            load_library().da2_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def da2_plan(B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float, frac4: float,
+             lam: float = 0.2, softmax_scale: float = 0.0, rank_scope: int = DA2_RANK_ROW,
+             g_q=None, g_k=None, g_v=None, tile_h: int = 8, tile_w: int = 8) -> Plan:
+    cfg = _Config(B, H, T, Hg, Wg, head_dim, tile_h, tile_w, frac16, frac8, frac4, lam, softmax_scale, rank_scope, 0,
+                  None, None, None)
+    keep = []
+    for name, arr in (("g_q", g_q), ("g_k", g_k), ("g_v", g_v)):
+        if arr is not None:
+            buf = (ctypes.c_float * (B * H))(*[float(x) for x in arr])
+            keep.append(buf)
+            setattr(cfg, name, ctypes.cast(buf, ctypes.POINTER(ctypes.c_float)))
+    out = ctypes.c_void_p()
+    rc = load_library().da2_plan(ctypes.byref(cfg), ctypes.byref(out))
+    if rc != 0:
+        raise Da2Error(rc, "da2_plan")
+    return Plan(out.value)
+
+
+def da2_plan_info(plan: Plan) -> PlanInfo:
+    info = PlanInfo()
+    rc = load_library().da2_plan_info(plan.handle, ctypes.byref(info))
+    if rc != 0:
+        raise Da2Error(rc, "da2_plan_info")
+    return info
+
+
+def _ptr(t) -> int:
+    return int(t.data_ptr())
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+def da2_prepare(plan: Plan, q, k, v, workspace, stream=None) -> None:
+    """q, k, v: CUDA bf16 [B,H,N,d] contiguous; workspace: CUDA uint8 tensor of plan.info.workspace_bytes."""
+    rc = load_library().da2_prepare(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_prepare")
+
+
+def da2_attention_fwd(plan: Plan, q, k, v, workspace, out, stream=None) -> None:
+    rc = load_library().da2_attention_fwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(workspace), _ptr(out),
+                                          _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_attention_fwd")
+
+
+def da2_device_status(plan: Plan, workspace, stream=None) -> int:
+    return int(load_library().da2_device_status(plan.handle, _ptr(workspace), _stream(stream)))
+
+
+def da2_last_launch_count(plan: Plan) -> int:
+    return int(load_library().da2_last_launch_count(plan.handle))
+
+
+def da2_plan_destroy(plan: Plan) -> None:
+    plan.close()
+
+
+def attention(plan: Plan, q, k, v, workspace=None, out=None, stream=None):
+    """Convenience: da2_prepare + da2_attention_fwd; allocates workspace / out through torch when not given."""
+    import torch
+    if not (q.is_cuda and k.is_cuda and v.is_cuda):
+        raise RuntimeError("da2 runs on CUDA tensors only (no CPU fallback)")
+    for t in (q, k, v):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("q, k, v must be contiguous bf16 [B,H,N,d]")
+    if workspace is None:
+        workspace = torch.empty(int(plan.info.workspace_bytes), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty_like(q)
+    da2_prepare(plan, q, k, v, workspace, stream)
+    da2_attention_fwd(plan, q, k, v, workspace, out, stream)
+    return out, workspace

@@ -1,0 +1,255 @@
+// C-ABI entry points of the da2 library: host-side plan (tiling, quotas, workspace layout) and the two device calls.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "da2_internal.cuh"
+
+namespace {
+
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  uint64_t cur = 0;
+  uint64_t take(uint64_t bytes) {
+    uint64_t off = cur;
+    cur = align_up(cur + bytes, 256);
+    return off;
+  }
+};
+
+// Integer quotas from fractions of M candidates (App. C.1: integer quotas T_p whose sum is the retained budget).
+// Cumulative round-half-up keeps the three counts consistent with the rounded total.
+void quotas_from_fractions(double f16, double f8, double f4, long long M, long long out[3]) {
+  long long c16 = (long long)std::floor(f16 * (double)M + 0.5);
+  long long c8 = (long long)std::floor((f16 + f8) * (double)M + 0.5);
+  long long c4 = (long long)std::floor((f16 + f8 + f4) * (double)M + 0.5);
+  c16 = c16 > M ? M : c16;
+  c8 = c8 > M ? M : c8;
+  c4 = c4 > M ? M : c4;
+  out[2] = c16;
+  out[1] = c8 - c16;
+  out[0] = c4 - c8;
+}
+
+da2::Params make_params(const da2_plan_t *plan, void *workspace) {
+  const da2_plan_info_t &I = plan->info;
+  da2::Params p;
+  std::memset(&p, 0, sizeof(p));
+  p.B = I.B; p.H = I.H; p.T = I.T; p.Hg = I.Hg; p.Wg = I.Wg; p.d = I.head_dim;
+  p.nty = I.nty; p.ntx = I.ntx; p.R_f = I.R_f; p.R = I.R; p.N = I.N; p.BH = I.B * I.H;
+  p.rank_scope = I.rank_scope;
+  for (int t = 0; t < 3; ++t) {
+    p.tier_active[t] = I.tier_active[t];
+    p.quota[t] = I.quota[t];
+    p.qrec_bytes[t] = I.qrec_bytes[t];
+    p.kvrec_bytes[t] = I.kvrec_bytes[t];
+  }
+  p.ids_per_head = I.ids_per_head;
+  p.lambda = I.lambda;
+  p.scale = I.softmax_scale;
+  uint8_t *w = (uint8_t *)workspace;
+  p.status = (int *)(w + I.off_status);
+  p.amax = (uint32_t *)(w + I.off_amax);
+  p.vmax = (uint32_t *)(w + I.off_vmax);
+  p.gscale = (float *)(w + I.off_gscale);
+  for (int i = 0; i < 4; ++i) p.desc[i] = (float *)(w + I.off_desc[i]);
+  for (int i = 0; i < 2; ++i) p.logits[i] = (float *)(w + I.off_logits[i]);
+  p.map = (float *)(w + I.off_map);
+  p.counts = (int *)(w + I.off_counts);
+  p.ids = (uint16_t *)(w + I.off_ids);
+  p.select = (uint32_t *)(w + I.off_select);
+  for (int t = 0; t < 3; ++t) {
+    p.qrec[t] = w + I.off_qrec[t];
+    p.kvrec[t] = w + I.off_kvrec[t];
+  }
+  p.dq8 = (float *)(w + I.off_dq8);
+  p.dk8 = (float *)(w + I.off_dk8);
+  p.dv8 = (float *)(w + I.off_dv8);
+  return p;
+}
+
+bool misaligned(const void *ptr, uintptr_t a) { return ((uintptr_t)ptr % a) != 0; }
+
+}  // namespace
+
+extern "C" {
+
+da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
+  if (!cfg || !plan_out) return DA2_ERR_INVALID_ARG;
+  *plan_out = nullptr;
+  if (cfg->B < 1 || cfg->H < 1 || cfg->T < 1 || cfg->Hg < 1 || cfg->Wg < 1) return DA2_ERR_INVALID_ARG;
+  if (cfg->frac16 < 0 || cfg->frac8 < 0 || cfg->frac4 < 0 || cfg->frac16 + cfg->frac8 + cfg->frac4 > 1.0 + 1e-12)
+    return DA2_ERR_INVALID_ARG;
+  if (!(cfg->lambda >= 0.0f && cfg->lambda <= 1.0f)) return DA2_ERR_INVALID_ARG;
+  if (cfg->rank_scope != DA2_RANK_ROW && cfg->rank_scope != DA2_RANK_HEAD) return DA2_ERR_INVALID_ARG;
+  if (cfg->reserved != 0) return DA2_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return DA2_ERR_UNSUPPORTED;
+  if (cfg->tile_h != 8 || cfg->tile_w != 8) return DA2_ERR_UNSUPPORTED;
+
+  da2_plan_t *plan = new (std::nothrow) da2_plan_t();
+  if (!plan) return DA2_ERR_INTERNAL;
+  plan->cfg = *cfg;
+  plan->last_launches = 0;
+  for (int i = 0; i < 3; ++i) plan->g_host[i] = nullptr;
+
+  da2_plan_info_t &I = plan->info;
+  std::memset(&I, 0, sizeof(I));
+  I.B = cfg->B; I.H = cfg->H; I.T = cfg->T; I.Hg = cfg->Hg; I.Wg = cfg->Wg; I.head_dim = cfg->head_dim;
+  I.tile_h = 8; I.tile_w = 8;
+  I.nty = (cfg->Hg + 7) / 8;
+  I.ntx = (cfg->Wg + 7) / 8;
+  I.R_f = I.nty * I.ntx;
+  long long R = (long long)cfg->T * I.R_f;
+  if (R > 16384) { delete plan; return DA2_ERR_UNSUPPORTED; }  // ids are uint16; row buffers live in shared memory
+  I.R = (int32_t)R;
+  I.S = da2::kSlots;
+  I.N = (int64_t)cfg->T * cfg->Hg * cfg->Wg;
+  I.rank_scope = cfg->rank_scope;
+  I.lambda = cfg->lambda;
+  I.softmax_scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  const long long M = cfg->rank_scope == DA2_RANK_ROW ? R : R * R;
+  long long qt[3];
+  quotas_from_fractions(cfg->frac16, cfg->frac8, cfg->frac4, M, qt);
+  for (int t = 0; t < 3; ++t) { I.quota[t] = qt[t]; I.tier_active[t] = qt[t] > 0; }
+
+  const uint64_t BH = (uint64_t)cfg->B * cfg->H, d = cfg->head_dim, S = da2::kSlots;
+  const long long kept = qt[0] + qt[1] + qt[2];
+  if (cfg->rank_scope == DA2_RANK_ROW) {
+    long long stride = (kept + 7) / 8 * 8;
+    if (stride == 0) stride = 8;
+    I.ids_per_head = stride * R;
+  } else {
+    I.ids_per_head = (kept + 7) / 8 * 8 + 8;
+  }
+
+  // record sizes: tier 0 NVFP4, tier 1 INT8/E4M3, tier 2 BF16
+  I.qrec_bytes[0] = (uint32_t)(S * d / 2 + (d / 64) * da2::kSfAtomBytes);
+  I.qrec_bytes[1] = (uint32_t)(S * d);
+  I.qrec_bytes[2] = (uint32_t)(S * d * 2);
+  I.kvrec_bytes[0] = (uint32_t)(S * d / 2 + (d / 64) * da2::kSfAtomBytes + d * S / 2 + da2::kSfAtomBytes);
+  I.kvrec_bytes[1] = (uint32_t)(2 * S * d);
+  I.kvrec_bytes[2] = (uint32_t)(4 * S * d);
+
+  Carver c;
+  I.off_status = c.take(64 * 4);
+  I.off_amax = c.take(BH * 4 * 4);
+  I.off_vmax = c.take(BH * d * 4);
+  I.off_gscale = c.take(BH * 4 * 4);
+  for (int i = 0; i < 4; ++i) I.off_desc[i] = c.take(BH * R * d * 4);
+  for (int i = 0; i < 2; ++i) I.off_logits[i] = c.take(BH * R * R * 4);
+  I.off_map = c.take(BH * R * R * 4);
+  I.off_counts = c.take(BH * R * 4 * 4);
+  I.off_ids = c.take(BH * (uint64_t)I.ids_per_head * 2);
+  I.off_select = c.take(BH * (4096 + 8 * (uint64_t)R) * 4);
+  for (int t = 0; t < 3; ++t) {
+    I.off_qrec[t] = c.take(I.tier_active[t] ? BH * R * I.qrec_bytes[t] : 0);
+    I.off_kvrec[t] = c.take(I.tier_active[t] ? BH * R * I.kvrec_bytes[t] : 0);
+  }
+  I.off_dq8 = c.take(BH * R * 4);
+  I.off_dk8 = c.take(BH * R * 4);
+  I.off_dv8 = c.take(BH * d * 4);
+  I.workspace_bytes = c.cur;
+
+  const float *src[3] = {cfg->g_q, cfg->g_k, cfg->g_v};
+  for (int i = 0; i < 3; ++i) {
+    if (!src[i]) continue;
+    plan->g_host[i] = (float *)std::malloc(BH * sizeof(float));
+    if (!plan->g_host[i]) { da2_plan_destroy(plan); return DA2_ERR_INTERNAL; }
+    for (uint64_t j = 0; j < BH; ++j) {
+      if (!(src[i][j] > 0.0f)) { da2_plan_destroy(plan); return DA2_ERR_INVALID_ARG; }
+      plan->g_host[i][j] = src[i][j];
+    }
+  }
+  plan->cfg.g_q = plan->g_host[0];
+  plan->cfg.g_k = plan->g_host[1];
+  plan->cfg.g_v = plan->g_host[2];
+  *plan_out = plan;
+  return DA2_OK;
+}
+
+da2_status_t da2_plan_info(const da2_plan_t *plan, da2_plan_info_t *info) {
+  if (!plan || !info) return DA2_ERR_INVALID_ARG;
+  *info = plan->info;
+  return DA2_OK;
+}
+
+da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
+                         size_t workspace_bytes, void *stream) {
+  if (!plan || !q || !k || !v || !workspace) return DA2_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(workspace, 256))
+    return DA2_ERR_INVALID_ARG;
+  if (workspace_bytes < plan->info.workspace_bytes) return DA2_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  da2::Params p = make_params(plan, workspace);
+  const da2_plan_info_t &I = plan->info;
+  int launches = 0;
+  plan->last_launches = 0;
+  // status word, head maxima and per-channel maxima start at zero (they are contiguous)
+  if (cudaMemsetAsync((uint8_t *)workspace + I.off_status, 0, I.off_gscale - I.off_status, st) != cudaSuccess)
+    return DA2_ERR_CUDA;
+  const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k, *vb = (const __nv_bfloat16 *)v;
+  if (da2::launch_pool(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  for (int i = 0; i < 3; ++i) {  // caller-fixed NVFP4 per-tensor scales replace the derived ones
+    if (!plan->g_host[i]) continue;
+    if (cudaMemcpy2DAsync(p.gscale + i, 4 * sizeof(float), plan->g_host[i], sizeof(float), sizeof(float),
+                          (size_t)p.BH, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return DA2_ERR_CUDA;
+  }
+  if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  if (da2::launch_prep(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  plan->last_launches = launches;
+  return DA2_OK;
+}
+
+da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                               const void *workspace, void *out, void *stream) {
+  if (!plan || !q || !k || !v || !workspace || !out) return DA2_ERR_INVALID_ARG;
+  if (misaligned(out, 16) || misaligned(workspace, 256)) return DA2_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return DA2_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  da2::Params p = make_params(plan, const_cast<void *>(workspace));
+  int launches = 0;
+  plan->last_launches = 0;
+  if (da2::launch_attention(p, (__nv_bfloat16 *)out, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  plan->last_launches = launches;
+  return DA2_OK;
+}
+
+da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, void *stream) {
+  if (!plan || !workspace) return DA2_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int word[4] = {0, 0, 0, 0};
+  if (cudaMemcpyAsync(word, (const uint8_t *)workspace + plan->info.off_status, sizeof(word),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return DA2_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DA2_ERR_CUDA;
+  if (word[0] == da2::kDevOk) return DA2_OK;
+  if (word[0] == da2::kDevTimeout) return DA2_ERR_TIMEOUT;
+  return DA2_ERR_INTERNAL;
+}
+
+int32_t da2_last_launch_count(const da2_plan_t *plan) { return plan ? plan->last_launches : 0; }
+
+void da2_plan_destroy(da2_plan_t *plan) {
+  if (!plan) return;
+  for (int i = 0; i < 3; ++i) std::free(plan->g_host[i]);
+  delete plan;
+}
+
+const char *da2_status_string(da2_status_t status) {
+  switch (status) {
+    case DA2_OK: return "ok";
+    case DA2_ERR_INVALID_ARG: return "invalid argument";
+    case DA2_ERR_UNSUPPORTED: return "unsupported configuration";
+    case DA2_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case DA2_ERR_CUDA: return "CUDA error";
+    case DA2_ERR_TIMEOUT: return "device-side wait timed out";
+    case DA2_ERR_INTERNAL: return "internal error";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

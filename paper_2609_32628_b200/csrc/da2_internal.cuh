@@ -1,0 +1,83 @@
+// Internal declarations shared by the da2 kernels (host plan, device parameter block, small helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "da2.h"
+
+namespace da2 {
+
+constexpr int kSlots = 64;      // tokens per block: one 8 x 8 spatial tile of one frame
+constexpr int kTile = 8;
+constexpr int kSfAtomBytes = 512;  // one scale-factor atom: 128 rows x 4 groups of E4M3 codes
+
+// device status word values (workspace off_status[0])
+constexpr int kDevOk = 0;
+constexpr int kDevTimeout = 1;
+constexpr int kDevBadList = 2;
+
+// Plain-old-data parameter block handed to every kernel by value.
+struct Params {
+  int B, H, T, Hg, Wg, d;
+  int nty, ntx, R_f, R;
+  long long N;
+  int BH;
+  int rank_scope;
+  int tier_active[3];       // 0: NVFP4, 1: INT8/E4M3, 2: BF16
+  long long quota[3];       // k4, k8, k16
+  long long ids_per_head;
+  float lambda, scale;
+  uint32_t qrec_bytes[3], kvrec_bytes[3];
+  // resolved device pointers into the workspace
+  int *status;
+  uint32_t *amax;           // [BH][4]
+  uint32_t *vmax;           // [BH][d]
+  float *gscale;            // [BH][4]
+  float *desc[4];           // Qavg, Qmax, Kavg, Kmax [BH][R][d]
+  float *logits[2];         // [BH][R][R]
+  float *map;               // [BH][R][R]
+  int *counts;              // [BH][R][4]
+  uint16_t *ids;            // [BH][ids_per_head]
+  uint32_t *select;         // HEAD-scope scratch
+  uint8_t *qrec[3], *kvrec[3];
+  float *dq8, *dk8, *dv8;
+};
+
+// number of valid rows / columns of tile (ty, tx) and the 64-bit slot-valid mask of block a
+__host__ __device__ inline unsigned long long block_valid_mask(const Params &p, int a) {
+  int r = a % p.R_f;
+  int ty = r / p.ntx, tx = r % p.ntx;
+  int vr = min(kTile, p.Hg - ty * kTile), vc = min(kTile, p.Wg - tx * kTile);
+  unsigned long long rowbits = (vc >= 8) ? 0xffull : ((1ull << vc) - 1ull);
+  unsigned long long m = 0;
+  for (int ly = 0; ly < vr; ++ly) m |= rowbits << (8 * ly);
+  return m;
+}
+
+// raster token index of slot j of block a (caller checks validity with the mask)
+__host__ __device__ inline long long slot_token(const Params &p, int a, int j) {
+  int t = a / p.R_f, r = a % p.R_f;
+  int ty = r / p.ntx, tx = r % p.ntx;
+  int y = ty * kTile + (j >> 3), x = tx * kTile + (j & 7);
+  return ((long long)t * p.Hg + y) * p.Wg + x;
+}
+
+// kernel launchers (each returns the cudaError_t of its launch)
+cudaError_t launch_pool(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
+                        cudaStream_t st, int *launches);
+cudaError_t launch_draft(const Params &p, cudaStream_t st, int *launches);
+cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches);
+cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
+                        cudaStream_t st, int *launches);
+cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);
+
+}  // namespace da2
+
+struct da2_plan {
+  da2_config_t cfg;
+  da2_plan_info_t info;
+  float *g_host[3];       // optional caller-provided NVFP4 per-tensor scales (copied), or nullptr
+  mutable int last_launches;
+};

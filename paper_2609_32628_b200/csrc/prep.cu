@@ -1,0 +1,247 @@
+// Kernel 3: fused operand preparation.  One pass over Q, K, V reorders every 8 x 8 spatial tile into a contiguous
+// block and quantises it to each active format (App. C.3), writing the result directly as the shared-memory image
+// the attention kernel streams in (K-major 8 x 16-byte core matrices, V already transposed to [channel][key slot],
+// scale factors in the layout the block-scaled tensor-core instruction reads) -- see da2.h for the record layout.
+//   INT8  Q/K : one fp32 scale per block, delta = amax/127 + 1e-7, round half away from zero
+//   E4M3  V   : per-(head, channel) scale delta_c = max|V_c| / 2.25
+//   NVFP4 Q/K : E2M1 with one E4M3 scale per 16 channels; V: per 16 key slots of a channel; per-head scale g_X
+//   BF16      : the stored values, reordered only
+// Every fp32 operation below is a single correctly rounded operation in the order the format definition gives, so
+// codes and scales are reproducible bit for bit.  HBM-bound: reads 3*64*d*2 bytes per block, writes the records.
+#include <cuda_fp8.h>
+
+#include "da2_internal.cuh"
+
+namespace da2 {
+
+namespace {
+
+constexpr int NT = 256;
+
+__device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+
+__device__ __forceinline__ uint32_t cast_e4m3(float x) {
+  return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
+}
+
+// two floats -> two E2M1 codes, `lo` in bits 3:0 and `hi` in bits 7:4 (round to nearest even, saturating)
+__device__ __forceinline__ uint32_t cast_e2m1x2(float lo, float hi) {
+  uint16_t r;
+  asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; mov.b16 %0, {t, 0}; }" : "=h"(r) : "f"(lo), "f"(hi));
+  return (uint32_t)r;
+}
+
+__device__ __forceinline__ float decode_e4m3(uint32_t c) {
+  const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3);
+  return __half2float(*reinterpret_cast<const __half *>(&h));
+}
+
+// NVFP4 group of 16 values (Eq. "v2-nvfp4-quantization"): returns the E4M3 scale code, writes 8 bytes of codes
+__device__ __forceinline__ uint32_t nvfp4_group(const float (&x)[16], float g, uint32_t (&packed)[2]) {
+  float gmax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) gmax = fmaxf(gmax, fabsf(x[i]));
+  const uint32_t sc = cast_e4m3(__fdiv_rn(gmax, __fmul_rn(6.0f, g)));
+  const float sigma = decode_e4m3(sc);
+  packed[0] = 0; packed[1] = 0;
+  if (sigma == 0.f) return sc;  // a group whose encoded scale is zero is encoded as zero
+  const float step = __fmul_rn(g, sigma);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t b = cast_e2m1x2(__fdiv_rn(x[2 * i], step), __fdiv_rn(x[2 * i + 1], step));
+    packed[i >> 2] |= b << (8 * (i & 3));
+  }
+  return sc;
+}
+
+template <int D>
+__global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 *__restrict__ q,
+                                                  const __nv_bfloat16 *__restrict__ k,
+                                                  const __nv_bfloat16 *__restrict__ v) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  uint16_t *tq = reinterpret_cast<uint16_t *>(smem);   // [64][D]
+  uint16_t *tk = tq + kSlots * D;
+  uint16_t *tv = tk + kSlots * D;
+  uint8_t *sf_img = reinterpret_cast<uint8_t *>(tv + kSlots * D);  // up to 3 atoms (Q or K: D/64, V: 1)
+  __shared__ float s_red[2][NT / 32];
+  __shared__ float s_delta[2];
+
+  const int a = blockIdx.x, bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned long long mask = block_valid_mask(p, a);
+  const size_t head_off = (size_t)bh * p.N * D;
+  const size_t blk = (size_t)bh * p.R + a;
+
+  // stage the three tiles, padding slots as zeros; track max|Q|, max|K| of the block
+  float aq = 0.f, ak = 0.f;
+  constexpr int CPR = D / 8;
+  for (int idx = tid; idx < kSlots * CPR; idx += NT) {
+    const int j = idx / CPR, c8 = idx % CPR;
+    uint4 xq = make_uint4(0, 0, 0, 0), xk = xq, xv = xq;
+    if ((mask >> j) & 1ull) {
+      const size_t off = head_off + (size_t)slot_token(p, a, j) * D + c8 * 8;
+      xq = *reinterpret_cast<const uint4 *>(q + off);
+      xk = *reinterpret_cast<const uint4 *>(k + off);
+      xv = *reinterpret_cast<const uint4 *>(v + off);
+    }
+    *reinterpret_cast<uint4 *>(tq + j * D + c8 * 8) = xq;
+    *reinterpret_cast<uint4 *>(tk + j * D + c8 * 8) = xk;
+    *reinterpret_cast<uint4 *>(tv + j * D + c8 * 8) = xv;
+    const uint32_t wq[4] = {xq.x, xq.y, xq.z, xq.w}, wk[4] = {xk.x, xk.y, xk.z, xk.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      aq = fmaxf(aq, fmaxf(fabsf(__uint_as_float(wq[i] << 16)), fabsf(__uint_as_float(wq[i] & 0xffff0000u))));
+      ak = fmaxf(ak, fmaxf(fabsf(__uint_as_float(wk[i] << 16)), fabsf(__uint_as_float(wk[i] & 0xffff0000u))));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    aq = fmaxf(aq, __shfl_xor_sync(0xffffffffu, aq, o));
+    ak = fmaxf(ak, __shfl_xor_sync(0xffffffffu, ak, o));
+  }
+  if (lane == 0) { s_red[0][warp] = aq; s_red[1][warp] = ak; }
+  __syncthreads();
+  if (tid < 2) {
+    float m = 0.f;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) m = fmaxf(m, s_red[tid][w]);
+    const float delta = __fadd_rn(__fdiv_rn(m, 127.0f), 1e-7f);
+    s_delta[tid] = delta;
+    if (p.tier_active[1]) (tid == 0 ? p.dq8 : p.dk8)[blk] = delta;
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ tier 2: BF16, reorder only
+  if (p.tier_active[2]) {
+    uint8_t *qr = p.qrec[2] + blk * p.qrec_bytes[2];
+    uint8_t *kr = p.kvrec[2] + blk * p.kvrec_bytes[2];
+    uint8_t *vr = kr + kSlots * D * 2;
+    for (int idx = tid; idx < kSlots * D / 8; idx += NT) {  // chunk (kc, r): channels kc*8.. of slot r
+      const int kc = idx / kSlots, r = idx % kSlots;
+      *reinterpret_cast<uint4 *>(qr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tq + r * D + kc * 8);
+      *reinterpret_cast<uint4 *>(kr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tk + r * D + kc * 8);
+    }
+    for (int idx = tid; idx < D * kSlots / 8; idx += NT) {  // chunk (kc, c): slots kc*8.. of channel c
+      const int kc = idx / D, c = idx % D;
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        w[i] = (uint32_t)tv[(kc * 8 + 2 * i) * D + c] | ((uint32_t)tv[(kc * 8 + 2 * i + 1) * D + c] << 16);
+      *reinterpret_cast<uint4 *>(vr + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+
+  // ------------------------------------------------------------------ tier 1: INT8 Q/K, E4M3 V
+  if (p.tier_active[1]) {
+    uint8_t *qr = p.qrec[1] + blk * p.qrec_bytes[1];
+    uint8_t *kr = p.kvrec[1] + blk * p.kvrec_bytes[1];
+    uint8_t *vr = kr + kSlots * D;
+    const float dq = s_delta[0], dk = s_delta[1];
+    for (int idx = tid; idx < kSlots * D / 16; idx += NT) {  // chunk (kc, r): channels kc*16.. of slot r
+      const int kc = idx / kSlots, r = idx % kSlots;
+      uint32_t wq[4] = {0, 0, 0, 0}, wk[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int cq = (int)roundf(__fdiv_rn(bf16_to_f32(tq[r * D + kc * 16 + i]), dq));
+        const int ck = (int)roundf(__fdiv_rn(bf16_to_f32(tk[r * D + kc * 16 + i]), dk));
+        wq[i >> 2] |= (uint32_t)(cq & 0xff) << (8 * (i & 3));
+        wk[i >> 2] |= (uint32_t)(ck & 0xff) << (8 * (i & 3));
+      }
+      *reinterpret_cast<uint4 *>(qr + (size_t)idx * 16) = make_uint4(wq[0], wq[1], wq[2], wq[3]);
+      *reinterpret_cast<uint4 *>(kr + (size_t)idx * 16) = make_uint4(wk[0], wk[1], wk[2], wk[3]);
+    }
+    for (int idx = tid; idx < D * kSlots / 16; idx += NT) {  // chunk (kc, c): slots kc*16.. of channel c
+      const int kc = idx / D, c = idx % D;
+      const float dv = p.dv8[(size_t)bh * D + c];
+      uint32_t w[4] = {0, 0, 0, 0};
+      if (dv > 0.f) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int slot = kc * 16 + i;
+          uint32_t code = 0;
+          if ((mask >> slot) & 1ull) code = cast_e4m3(__fdiv_rn(bf16_to_f32(tv[slot * D + c]), dv));
+          w[i >> 2] |= code << (8 * (i & 3));
+        }
+      }
+      *reinterpret_cast<uint4 *>(vr + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+
+  // ------------------------------------------------------------------ tier 0: NVFP4
+  if (p.tier_active[0]) {
+    const float gq = p.gscale[bh * 4 + 0], gk = p.gscale[bh * 4 + 1], gv = p.gscale[bh * 4 + 2];
+    constexpr int QK_IMG = kSlots * D / 2, NATOM = D / 64;
+    uint8_t *qr = p.qrec[0] + blk * p.qrec_bytes[0];
+    uint8_t *kr = p.kvrec[0] + blk * p.kvrec_bytes[0];
+    uint8_t *vr = kr + QK_IMG + NATOM * kSfAtomBytes;
+    for (int which = 0; which < 2; ++which) {  // 0: Q, 1: K
+      const uint16_t *src = which ? tk : tq;
+      uint8_t *dst = which ? kr : qr;
+      const float g = which ? gk : gq;
+      __syncthreads();
+      for (int i = tid; i < NATOM * kSfAtomBytes / 4; i += NT) reinterpret_cast<uint32_t *>(sf_img)[i] = 0;
+      __syncthreads();
+      for (int idx = tid; idx < kSlots * D / 32; idx += NT) {  // chunk (kc, r): channels kc*32.. of slot r
+        const int kc = idx / kSlots, r = idx % kSlots;
+        uint32_t w[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float x[16];
+          uint32_t pk[2];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(src[r * D + kc * 32 + h * 16 + i]);
+          const uint32_t sc = nvfp4_group(x, g, pk);
+          w[2 * h] = pk[0]; w[2 * h + 1] = pk[1];
+          const int grp = kc * 2 + h;  // 16-channel group index; 4 groups per atom
+          sf_img[(grp >> 2) * kSfAtomBytes + (r & 31) * 16 + (r >> 5) * 4 + (grp & 3)] = (uint8_t)sc;
+        }
+        *reinterpret_cast<uint4 *>(dst + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      __syncthreads();
+      for (int i = tid; i < NATOM * kSfAtomBytes / 16; i += NT)
+        *reinterpret_cast<uint4 *>(dst + QK_IMG + (size_t)i * 16) = reinterpret_cast<const uint4 *>(sf_img)[i];
+    }
+    __syncthreads();
+    for (int i = tid; i < kSfAtomBytes / 4; i += NT) reinterpret_cast<uint32_t *>(sf_img)[i] = 0;
+    __syncthreads();
+    for (int idx = tid; idx < D * kSlots / 32; idx += NT) {  // chunk (kc, c): slots kc*32.. of channel c
+      const int kc = idx / D, c = idx % D;
+      uint32_t w[4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float x[16];
+        uint32_t pk[2];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(tv[(kc * 32 + h * 16 + i) * D + c]);
+        const uint32_t sc = nvfp4_group(x, gv, pk);
+        w[2 * h] = pk[0]; w[2 * h + 1] = pk[1];
+        sf_img[(c & 31) * 16 + (c >> 5) * 4 + (kc * 2 + h)] = (uint8_t)sc;
+      }
+      *reinterpret_cast<uint4 *>(vr + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __syncthreads();
+    for (int i = tid; i < kSfAtomBytes / 16; i += NT)
+      *reinterpret_cast<uint4 *>(vr + D * kSlots / 2 + (size_t)i * 16) = reinterpret_cast<const uint4 *>(sf_img)[i];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
+                        cudaStream_t st, int *launches) {
+  dim3 grid(p.R, p.BH);
+  const size_t smem = 3 * (size_t)kSlots * p.d * 2 + 3 * kSfAtomBytes;
+  cudaError_t e;
+  if (p.d == 128) {
+    e = cudaFuncSetAttribute(prep_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    prep_kernel<128><<<grid, NT, smem, st>>>(p, q, k, v);
+  } else {
+    e = cudaFuncSetAttribute(prep_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    prep_kernel<64><<<grid, NT, smem, st>>>(p, q, k, v);
+  }
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace da2
