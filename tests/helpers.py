@@ -16,11 +16,11 @@ def scale_of(w) -> float:
     return float(np.float32(1.0) / np.sqrt(np.float32(w.head_dim)))
 
 
-def run_gpu(w, q, k, v, rank_scope=0, lam=None):
+def run_gpu(w, q, k, v, rank_scope=0, lam=None, zero_ws=False):
     """q,k,v CUDA bf16 [B,H,N,d].  Returns (plan, workspace uint8 tensor, out)."""
     plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4,
                         lam=w.lam if lam is None else lam, rank_scope=rank_scope)
-    ws = torch.empty(int(plan.info.workspace_bytes), dtype=torch.uint8, device=q.device)
+    ws = (torch.zeros if zero_ws else torch.empty)(int(plan.info.workspace_bytes), dtype=torch.uint8, device=q.device)
     out = torch.full_like(q, float("nan"))
     da2.da2_prepare(plan, q, k, v, ws)
     da2.da2_attention_fwd(plan, q, k, v, ws, out)
