@@ -126,6 +126,29 @@ da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, vo
 /* Number of kernels the last da2_prepare / da2_attention_fwd call on this plan enqueued (for launch accounting). */
 int32_t da2_last_launch_count(const da2_plan_t *plan);
 
+/*
+ * Draft attention map without any device allocation or caller workspace (the paper has no counterpart: this is a
+ * packaging variant of the draft-map step for callers that cannot allocate).
+ *
+ * Who needs it: code that must not call cudaMalloc -- e.g. a serving loop where an allocation would stall the device,
+ * or a component whose device memory is owned and fully handed out by someone else -- and therefore cannot provide
+ * the workspace da2_prepare wants.  The scratch for the two branches' draft logits lives in a fixed device array
+ * inside the library (8 MiB, held by every GPU that loads the library until the process exits).
+ *
+ *   q_avg, q_max, k_avg, k_max : DEVICE, fp32 [BH][R][head_dim], 16-byte aligned (region descriptors, inputs)
+ *   map_out                    : DEVICE, fp32 [BH][R][R] (output, rows sum to 1)
+ *   limit                      : BH*R*R <= 1,048,576 and R <= 16384, head_dim a multiple of 16; larger problems
+ *                                return DA2_ERR_WORKSPACE_TOO_SMALL and launch nothing
+ * The first call on each device looks up the array's device address (with that device current); make that first
+ * call outside any stream capture.  All calls on a device share the array, which keeps the previous call's
+ * contents; every entry a call reads is written by that call first, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, no ordering) race on it: order them.
+ * Calls no cudaMalloc / cudaFree / allocating library routine.  Enqueues on stream, does not synchronise.
+ */
+da2_status_t da2_draft_map_noalloc(const float *q_avg, const float *q_max, const float *k_avg, const float *k_max,
+                                   int32_t BH, int32_t R, int32_t head_dim, float lambda, float softmax_scale,
+                                   float *map_out, void *stream);
+
 void da2_plan_destroy(da2_plan_t *plan);
 const char *da2_status_string(da2_status_t status);
 

@@ -163,6 +163,22 @@ def da2_plan_destroy(plan: Plan) -> None:
     plan.close()
 
 
+def da2_draft_map_noalloc(q_avg, q_max, k_avg, k_max, lam: float, softmax_scale: float, map_out, stream=None) -> None:
+    """Draft map from fp32 CUDA descriptors [BH,R,d] into map_out [BH,R,R] with no device allocation: for callers
+    that may not allocate device memory (the scratch is a fixed array inside the library, BH*R*R <= 2**20)."""
+    lib = load_library()
+    fn = lib.da2_draft_map_noalloc
+    fn.restype = ctypes.c_int
+    vp = ctypes.c_void_p
+    fn.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_float,
+                   vp, vp]
+    BH, R, d = q_avg.shape
+    rc = fn(_ptr(q_avg), _ptr(q_max), _ptr(k_avg), _ptr(k_max), BH, R, d, lam, softmax_scale, _ptr(map_out),
+            _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_draft_map_noalloc")
+
+
 def attention(plan: Plan, q, k, v, workspace=None, out=None, stream=None):
     """Convenience: da2_prepare + da2_attention_fwd; allocates workspace / out through torch when not given."""
     import torch

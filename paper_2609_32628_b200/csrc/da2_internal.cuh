@@ -69,6 +69,7 @@ cudaError_t launch_pool(const Params &p, const __nv_bfloat16 *q, const __nv_bflo
                         cudaStream_t st, int *launches);
 cudaError_t launch_draft(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches);
+cudaError_t launch_map_rows(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches);
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);

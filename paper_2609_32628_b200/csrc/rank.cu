@@ -398,6 +398,20 @@ __global__ void __launch_bounds__(NT) head_emit_kernel(Params p, int mode) {
 
 }  // namespace
 
+// Draft map rows only (softmax of both logit branches and their mixture into p.map); used by callers that want
+// the map without the ranking.
+cudaError_t launch_map_rows(const Params &p, cudaStream_t st, int *launches) {
+  dim3 grid(p.R, p.BH);
+  const size_t smem = (size_t)p.R * sizeof(uint32_t);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(head_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  head_map_kernel<<<grid, NT, smem, st>>>(p);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
 cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches) {
   dim3 grid(p.R, p.BH);
   const size_t smem = (size_t)p.R * sizeof(uint32_t);
