@@ -101,7 +101,7 @@ typedef struct {
  *             tier 1: image of E4M3 V^T [d x 64]
  *             tier 0: image of packed E2M1 V^T [d x 32 bytes], then one 512 B scale atom
  *   Packed E2M1: element 2i in the low nibble of byte i.  Scale atom (E4M3 codes, one per 16 elements along the
- *   reduction dimension): byte (row%32)*16 + (row/32)*4 + group, rows >= 64 unused for Q/K.
+ *   reduction dimension): byte (row%32)*16 + (row/32)*4 + group; Q/K atoms repeat rows 0..63 as rows 64..127.
  *   Padding slots of ragged edge tiles hold zeros.
  */
 

@@ -1,25 +1,35 @@
 // Kernel 4: phased mixed-precision block-sparse attention (Sec. 3.3 "Phased execution" and "Cross-precision
 // accumulation", App. C.3 / C.4).
 //
-// One CTA owns one query block (64 tokens) and walks its list: NVFP4 segment, then INT8/E4M3 segment, then BF16
-// segment.  All segments share the fp32 running row maximum h, the fp32 denominator l (which always sums the
-// exponential weights BEFORE they are converted to a matrix operand) and ONE output accumulator in tensor memory;
-// at a segment boundary the accumulator only changes units (Eq. "precision-state-conversion"), and the output is
-// normalised once at the end.
+// Every query block (64 tokens) walks its own list: NVFP4 segment, then INT8/E4M3 segment, then BF16 segment.  All
+// segments share the fp32 running row maximum h, the fp32 denominator l (which always sums the exponential weights
+// BEFORE they are converted to a matrix operand) and ONE output accumulator in tensor memory; at a segment boundary
+// the accumulator only changes units (Eq. "precision-state-conversion"), and the output is normalised once.
 //
-// Mapping onto sm_100a:
-//   S   = Q K^T   : tcgen05.mma, M = 128 (rows 0..63 are the block's queries, rows 64..127 are don't-care rows the
-//                   block-scaled instruction shape requires), N = 64 keys, K = d; fp32 / int32 accumulator in TMEM.
-//   O^T = V^T P^T : tcgen05.mma, M = 128 (channels; d = 64 leaves rows 64..127 unused), N = 64 queries, K = 64 keys.
-//                   Keeping O transposed makes the online-softmax correction a per-COLUMN scale, so only the queries
-//                   whose maximum moved are touched, and makes the per-channel unit changes a per-lane scalar.
-//   kinds         : kind::f16 (BF16), kind::i8 for QK^T + kind::f8f6f4 (E4M3 x E4M3) for PV (App. C.1: the INT8 path
-//                   uses INT8 for QK^T and FP8 for PV), kind::mxf4nvf4 with E4M3 scales per 16 elements (NVFP4).
-//   operands      : da2_prepare wrote every block as a ready shared-memory image, so one 1-D bulk copy per step
-//                   brings K, V^T and their scale factors; P and its NVFP4 scale factors are produced by the softmax
-//                   threads into shared memory (tcgen05.cp moves scale factors into TMEM).
-// Every wait on an mbarrier is bounded; a wait that gives up records DA2 device status "timeout" and the CTA winds
-// down normally (TMEM released).
+// Mapping onto sm_100a
+//   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 512 threads in four roles:
+//     warps 0-7   softmax: stream = (warp%4)/2, two threads per query row (32 of the 64 key columns each); they read
+//                 S from TMEM, keep h and a partial l, and write P~ (and its NVFP4 scale factors) to shared memory
+//     warps 8-11  correction + epilogue: rescale the accumulator columns of queries whose maximum moved, apply the
+//                 per-channel unit change at a segment boundary, and finally normalise, transpose and store
+//     warps 12,13 MMA issue, one thread per stream: S = Q K^T and O^T += V^T P~^T with tcgen05.mma, accumulators
+//                 in TMEM.  This thread's instruction count is on the critical path of every step, so its operand
+//                 descriptors are built once and only offset inside the loop
+//     warps 14,15 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings
+//   S   = Q K^T   : M = 128, N = 64 keys, K = d.  The block-scaled instruction only exists at M = 128, so stream 0's
+//                   queries sit in rows 0..63 and stream 1's in rows 64..127 (its operand descriptor starts 1 KB
+//                   early); the other 64 rows of each product are don't-care.  S is double buffered.
+//   O^T = V^T P^T : M = 128 channels, N = 64 queries, K = 64 keys.  Keeping O transposed makes the online-softmax
+//                   correction a per-COLUMN scale, so only queries whose maximum moved are touched, and makes the
+//                   per-channel unit changes (eta*delta_c^V, g_V/2688) per-lane scalars.
+//   kinds         : kind::f16 (BF16); kind::i8 for QK^T + kind::f8f6f4 E4M3 x E4M3 for PV (App. C.1); and
+//                   kind::mxf4nvf4 with E4M3 scales per 16 elements (NVFP4), scale factors moved by tcgen05.cp.
+// The softmax is the bound (one ex2 per score on a 16-lane/clk unit), so its inner loops are written to spend as few
+// issue slots per score as possible: the row maximum is taken on raw accumulator values, the scale and the maximum
+// are folded into one FMA feeding ex2, int32 scores become floats through a magic-number add folded into that FMA,
+// and the NVFP4 group scale is folded into the exponent so the scaled weight needs no extra multiply.
+// Every wait on an mbarrier is bounded; a wait that gives up records device status "timeout", all roles leave their
+// loops and the CTA exits normally after releasing TMEM.
 #include <cuda_fp8.h>
 
 #include "da2_internal.cuh"
@@ -29,44 +39,95 @@ namespace da2 {
 
 namespace {
 
-constexpr int NT = 128;
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t COL_S = 0, COL_O = 64, COL_SFQ = 128, COL_SFK = 136, COL_SFV = 144, COL_SFP = 148;
+constexpr int kSoftmaxWarps = 8, kCorrWarps = 4;
+constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // warps 12, 13: MMA issue for stream 0, 1
+constexpr int kLoadWarp0 = kMmaWarp0 + 2;              // warps 14, 15: loader for stream 0, 1
+constexpr int NT = (kLoadWarp0 + 2) * 32;              // 512
+constexpr uint32_t kTmemCols = 512;
+// TMEM column map
+__host__ __device__ constexpr uint32_t col_s(int s, int buf) { return (uint32_t)(s * 2 + buf) * 64u; }
+__host__ __device__ constexpr uint32_t col_o(int s) { return 256u + (uint32_t)s * 64u; }
+// scale factors: every region starts on a multiple of 4 columns (one 4-column group holds 128 rows x 4 scales)
+__host__ __device__ constexpr uint32_t col_sfq(int s) { return 384u + (uint32_t)s * 8u; }  // 4 columns per K step
+__host__ __device__ constexpr uint32_t col_sfk(int s) { return 400u + (uint32_t)s * 8u; }
+__host__ __device__ constexpr uint32_t col_sfv(int s) { return 416u + (uint32_t)s * 4u; }
+__host__ __device__ constexpr uint32_t col_sfp(int s) { return 424u + (uint32_t)s * 4u; }
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kEtaP8 = 0.0022326917f;  // probability dequantisation scale of the 8-bit path
 constexpr float kOffsetP8 = 8.807f;      // base-2 exponent offset (about log2 448)
+constexpr int kWindow = 64;              // list entries the loader stages at a time
+
+// barrier indices inside one stream's group
+// (a parity wait can only tell the latest completion from the one before, so every barrier is laid out such that no
+// waiter can fall two completions behind: buffers indexed by step parity get one barrier per buffer)
+enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_FREADY = 22,
+       B_XREADY = 24, B_PVDONE = 26, B_OCORR = 28, B_ELL = 30, B_Q = 31, B_COUNT = 32 };
+constexpr int kMaxStages = 4, kInfoRing = 8;
 
 struct SmemMap {
-  uint32_t q[3];     // Q record per tier (only active tiers are resident)
-  uint32_t kv[2];    // two K/V stages
-  uint32_t p;        // P operand image, 64 x 64 x <= 2 bytes
-  uint32_t sfp;      // P scale atom (512 B)
-  uint32_t factor;   // 64 floats: per-query correction factor of this step
-  uint32_t inv_l;    // 64 floats
-  uint32_t changed;  // 64 bytes: 1 if the query's maximum moved this step
-  uint32_t bars;     // mbarriers
+  uint32_t q[2][3];   // Q record per stream and tier
+  uint32_t kst[2][kMaxStages];  // K ring per stream (K image + its scale atoms)
+  uint32_t vst[2][kMaxStages];  // V ring per stream (V^T image + its scale atom)
+  int nk, nv;                   // ring depths
+  uint32_t kbytes[3], vbytes[3];
+  uint32_t p[2][2];   // P operand images per stream, double buffered (64 x 64 x <= 2 bytes)
+  uint32_t sfp[2][2]; // P scale atoms (512 B)
+  uint32_t factor;    // float [2 streams][2][64]
+  uint32_t changed;   // uint8 [2][2][64]
+  uint32_t xmax;      // float [2][2 parity][2 halves][64]
+  uint32_t ell;       // float [2][2 halves][64]
+  uint32_t info;      // per stream, ring of kInfoRing steps: {u64 mask, float dk8, pad}
+  uint32_t win;       // loader window: per stream ids u16[256], dk f32[256], mask u64[256]
+  uint32_t bars;      // uint64 [2][B_COUNT]
+  uint32_t kstage, vstage;  // bytes per ring stage
+  uint32_t chg;             // uint32 [2 streams][2][2]: ballots of the queries whose maximum moved this step
   uint32_t total;
-  uint32_t kv_bytes;
 };
 
 __host__ SmemMap make_smem_map(const Params &p) {
   SmemMap m;
   uint32_t cur = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = cur; cur = (cur + bytes + 127u) / 128u * 128u; return o; };
-  for (int t = 0; t < 3; ++t) m.q[t] = p.tier_active[t] ? take(p.qrec_bytes[t]) : 0;
-  uint32_t kvb = 0;
-  for (int t = 0; t < 3; ++t)
-    if (p.tier_active[t] && p.kvrec_bytes[t] > kvb) kvb = p.kvrec_bytes[t];
-  if (kvb < 16384) kvb = 16384;  // stage 0 doubles as the output staging tile [64][d] bf16
-  m.kv_bytes = kvb;
-  m.kv[0] = take(kvb);
-  m.kv[1] = take(kvb);
-  m.p = take(8192);
-  m.sfp = take(512);
-  m.factor = take(256);
-  m.inv_l = take(256);
-  m.changed = take(64);
-  m.bars = take(64);
+  // stream 1's Q descriptors start 1 KB before its images: stream 0's records precede them, so that is valid memory
+  for (int s = 0; s < 2; ++s)
+    for (int t = 0; t < 3; ++t) m.q[s][t] = p.tier_active[t] ? take(p.qrec_bytes[t]) : 0;
+  uint32_t kstage = 0, vstage = 0;
+  for (int t = 0; t < 3; ++t) {
+    m.kbytes[t] = p.qrec_bytes[t];                     // the K part of a record is laid out like a Q record
+    m.vbytes[t] = p.kvrec_bytes[t] - p.qrec_bytes[t];
+    if (p.tier_active[t]) { kstage = max(kstage, m.kbytes[t]); vstage = max(vstage, m.vbytes[t]); }
+  }
+  kstage = (kstage + 127u) / 128u * 128u;
+  vstage = (vstage + 127u) / 128u * 128u;
+  const uint32_t q_end = cur;
+  const uint32_t pbytes = p.tier_active[2] ? 8192u : (p.tier_active[1] ? 4096u : 2048u);
+  // ring depths: as deep as shared memory allows (the K ring also serves as the 16 KB output staging tile)
+  const uint32_t fixed = 4 * pbytes + 4 * 512 + 1024 + 256 + 2048 + 1024 + 2 * kInfoRing * 16 +
+                         2 * (kWindow * 14) + 2 * B_COUNT * 8 + 1024;
+  const uint32_t budget = 232448u - q_end - fixed;
+  const int cand[5][2] = {{4, 4}, {3, 4}, {3, 3}, {2, 3}, {2, 2}};
+  m.nk = 2; m.nv = 2;
+  for (int c = 0; c < 5; ++c) {
+    if (2u * (cand[c][0] * kstage + cand[c][1] * vstage) <= budget) { m.nk = cand[c][0]; m.nv = cand[c][1]; break; }
+  }
+  while ((uint32_t)m.nk * kstage < 16384u) kstage += 128u;
+  m.kstage = kstage; m.vstage = vstage;
+  for (int s = 0; s < 2; ++s) {
+    for (int g = 0; g < kMaxStages; ++g) m.kst[s][g] = g < m.nk ? take(kstage) : 0;
+  }
+  for (int s = 0; s < 2; ++s)
+    for (int g = 0; g < kMaxStages; ++g) m.vst[s][g] = g < m.nv ? take(vstage) : 0;
+  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.p[s][g] = take(pbytes);
+  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.sfp[s][g] = take(512);
+  m.factor = take(2 * 2 * 64 * 4);
+  m.changed = take(2 * 2 * 64);
+  m.chg = take(2 * 2 * 2 * 4);
+  m.xmax = take(2 * 2 * 2 * 64 * 4);
+  m.ell = take(2 * 2 * 64 * 4);
+  m.info = take(2 * kInfoRing * 16);
+  m.win = take(2 * (kWindow * 2 + kWindow * 4 + kWindow * 8));
+  m.bars = take(2 * B_COUNT * 8);
   m.total = cur;
   return m;
 }
@@ -74,6 +135,11 @@ __host__ SmemMap make_smem_map(const Params &p) {
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -86,10 +152,14 @@ __device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return (uint32_t)r;
 }
-__device__ __forceinline__ uint32_t pack_e2m1x2(float lo, float hi) {
-  uint16_t r;
-  asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; mov.b16 %0, {t, 0}; }" : "=h"(r) : "f"(lo), "f"(hi));
-  return (uint32_t)r;
+// four floats -> four E2M1 codes in the low 16 bits (x0 in bits 3:0)
+__device__ __forceinline__ uint32_t pack_e2m1x4(float x0, float x1, float x2, float x3) {
+  uint32_t r;
+  asm("{ .reg .b8 a, b; cvt.rn.satfinite.e2m1x2.f32 a, %2, %1; cvt.rn.satfinite.e2m1x2.f32 b, %4, %3; "
+      "mov.b32 %0, {a, b, 0, 0}; }"
+      : "=r"(r)
+      : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
+  return r;
 }
 __device__ __forceinline__ float decode_e4m3(uint32_t c) {
   const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3);
@@ -97,61 +167,102 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
 }
 
 // bounded wait that also gives up as soon as another thread of the CTA has flagged a failure
+// (the flag then holds 1 + the shared-memory offset of the barrier that was never completed, for diagnosis)
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-  for (uint32_t i = 0; i < (1u << 22); ++i) {
+  if (tc::mbar_try_wait(bar, parity)) return true;
+  // The hand-offs between roles are on the critical path of every step, so the wait polls without sleeping (a
+  // sleep costs far more than a hand-off); the bound is on elapsed clock cycles.
+  const long long t0 = clock64();
+  for (uint32_t i = 1;; ++i) {
     if (tc::mbar_try_wait(bar, parity)) return true;
-    if (i > 32) {
-      __nanosleep(128);
+    if ((i & 255u) == 0u) {
       if (*abort_flag) return false;
+      if (clock64() - t0 > 400000000ll) break;  // about 0.2 s
     }
   }
+  atomicCAS(const_cast<int *>(abort_flag), 0, 1 + (int)(tc::smem_u32(bar) & 0xffff));
   return false;
 }
 
+struct StreamInfo {
+  int a;         // query block, or -1
+  int n4, n48;   // end of the NVFP4 segment, end of the INT8 segment (list positions)
+  int L;
+  const uint16_t *ids;
+  __device__ __forceinline__ int tier(int i) const { return i < n4 ? 0 : (i < n48 ? 1 : 2); }
+};
+
+__device__ __forceinline__ StreamInfo load_stream(const Params &p, int bh, int a) {
+  StreamInfo st;
+  st.a = a < p.R ? a : -1;
+  st.n4 = st.n48 = st.L = 0;
+  st.ids = nullptr;
+  if (a < p.R) {
+    const int4 c = *reinterpret_cast<const int4 *>(p.counts + ((size_t)bh * p.R + a) * 4);
+    st.n4 = c.x; st.n48 = c.x + c.y; st.L = c.x + c.y + c.z;
+    st.ids = p.ids + (size_t)bh * p.ids_per_head + c.w;
+  }
+  return st;
+}
+
 template <int D>
-__global__ void __launch_bounds__(NT) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
+__global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int bh = blockIdx.x / p.R, a = blockIdx.x % p.R;
-  const int R = p.R;
-  const int *cnt = p.counts + ((size_t)bh * R + a) * 4;
-  const int n4 = cnt[0], n8 = cnt[1], n16 = cnt[2];
-  const int L = n4 + n8 + n16;
-  const uint16_t *ids = p.ids + (size_t)bh * p.ids_per_head + cnt[3];
-  const unsigned long long qmask = block_valid_mask(p, a);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int R = p.R, pairs = (R + 1) / 2;
+  const int bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
   __nv_bfloat16 *out_head = out + (size_t)bh * p.N * D;
+  const StreamInfo st0 = load_stream(p, bh, 2 * pr), st1 = load_stream(p, bh, 2 * pr + 1);
 
-  if (L == 0) {  // no retained key: the rows return zero (App. C.1)
-    for (int idx = tid; idx < kSlots * (D / 8); idx += NT) {
+  auto store_zero_rows = [&](int a, int first, int nthreads) {  // rows without a retained key return zero (App. C.1)
+    const unsigned long long qmask = block_valid_mask(p, a);
+    for (int idx = first; idx < kSlots * (D / 8); idx += nthreads) {
       const int j = idx / (D / 8), c8 = idx % (D / 8);
       if ((qmask >> j) & 1ull)
         *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, a, j) * D + c8 * 8) = make_uint4(0, 0, 0, 0);
     }
+  };
+  if (st0.L == 0 && st1.L == 0) {
+    if (st0.a >= 0) store_zero_rows(st0.a, tid, NT);
+    if (st1.a >= 0) store_zero_rows(st1.a, tid, NT);
     return;
   }
 
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + sm.bars);
-  uint64_t *bar_full = bars;      // [2]
-  uint64_t *bar_q = bars + 2;
-  uint64_t *bar_s = bars + 3;
-  uint64_t *bar_o = bars + 4;
-  float *s_factor = reinterpret_cast<float *>(smem + sm.factor);
-  float *s_inv_l = reinterpret_cast<float *>(smem + sm.inv_l);
-  uint8_t *s_changed = smem + sm.changed;
+  auto bar = [&](int s, int which) -> uint64_t * { return bars + s * B_COUNT + which; };
+  float *s_factor = reinterpret_cast<float *>(smem + sm.factor);      // [s][buf][64]
+  uint32_t *s_chg = reinterpret_cast<uint32_t *>(smem + sm.chg);      // [s][buf][2]
+  float *s_xmax = reinterpret_cast<float *>(smem + sm.xmax);          // [s][parity][half][64]
+  float *s_ell = reinterpret_cast<float *>(smem + sm.ell);            // [s][half][64]
+  uint8_t *s_info = smem + sm.info;                                   // [s][kInfoRing] 16 bytes
 
   if (warp == 0) {
     tc::tmem_alloc(&s_tmem_base, kTmemCols);
     tc::tmem_relinquish();
   }
-  if (tid == 0) {
-    tc::mbar_init(&bar_full[0], 1);
-    tc::mbar_init(&bar_full[1], 1);
-    tc::mbar_init(bar_q, 1);
-    tc::mbar_init(bar_s, 1);
-    tc::mbar_init(bar_o, 1);
+  if (tid == 32) {
+    for (int s = 0; s < 2; ++s) {
+      for (int g = 0; g < 2; ++g) {
+        tc::mbar_init(bar(s, B_SREADY + g), 1);
+        tc::mbar_init(bar(s, B_SFREE + g), 128);
+        tc::mbar_init(bar(s, B_PREADY + g), 128);
+        tc::mbar_init(bar(s, B_FREADY + g), 64);
+        tc::mbar_init(bar(s, B_XREADY + g), 128);
+        tc::mbar_init(bar(s, B_PVDONE + g), 1);
+        tc::mbar_init(bar(s, B_OCORR + g), 128);
+      }
+      for (int g = 0; g < kMaxStages; ++g) {
+        tc::mbar_init(bar(s, B_FULLK + g), 1);
+        tc::mbar_init(bar(s, B_FULLV + g), 1);
+        tc::mbar_init(bar(s, B_KFREE + g), 1);
+        tc::mbar_init(bar(s, B_VFREE + g), 1);
+      }
+      tc::mbar_init(bar(s, B_ELL), 128);
+      tc::mbar_init(bar(s, B_Q), 1);
+    }
     tc::fence_barrier_init();
     s_abort = 0;
   }
@@ -159,269 +270,388 @@ __global__ void __launch_bounds__(NT) attention_kernel(Params p, SmemMap sm, __n
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem = s_tmem_base;
+  volatile int *abortp = &s_abort;
 
-  auto tier_of_step = [&](int i) { return i < n4 ? 0 : (i < n4 + n8 ? 1 : 2); };
-  auto issue_kv = [&](int i) {  // thread 0 only
-    const int t = tier_of_step(i);
-    int b = ids[i];
-    if (b >= R) { atomicExch(p.status, kDevBadList); b = 0; }
-    const uint8_t *src = p.kvrec[t] + ((size_t)bh * R + b) * p.kvrec_bytes[t];
-    tc::mbar_arrive_expect_tx(&bar_full[i & 1], p.kvrec_bytes[t]);
-    tc::bulk_g2s(smem + sm.kv[i & 1], src, p.kvrec_bytes[t], &bar_full[i & 1]);
-  };
-
-  if (tid == 0) {
-    uint32_t qbytes = 0;
-    const int nn[3] = {n4, n8, n16};
-    for (int t = 0; t < 3; ++t) if (nn[t] > 0) qbytes += p.qrec_bytes[t];
-    tc::mbar_arrive_expect_tx(bar_q, qbytes);
-    for (int t = 0; t < 3; ++t)
-      if (nn[t] > 0)
-        tc::bulk_g2s(smem + sm.q[t], p.qrec[t] + ((size_t)bh * R + a) * p.qrec_bytes[t], p.qrec_bytes[t], bar_q);
-    issue_kv(0);
-    if (L > 1) issue_kv(1);
-  }
-
-  // per-row online-softmax state (threads 0..63 own query rows; log2 domain)
-  float h2 = -INFINITY, ell = 0.f;
-  const float gq = p.gscale[bh * 4 + 0], gk = p.gscale[bh * 4 + 1], gv = p.gscale[bh * 4 + 2];
-  const float dq8 = p.tier_active[1] ? p.dq8[(size_t)bh * R + a] : 0.f;
-  const float dv8 = (p.tier_active[1] && tid < D) ? p.dv8[(size_t)bh * D + tid] : 0.f;
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-  auto unit_of = [&](int t) -> float {  // common units per accumulator unit, for this thread's channel
-    return t == 0 ? __fdiv_rn(gv, 2688.0f) : (t == 1 ? kEtaP8 * dv8 : 1.0f);
-  };
-  int prev_tier = -1;
-  bool failed = false;
-
-  if (!wait_or_abort(bar_q, 0, &s_abort)) { s_abort = 1; failed = true; }
-  if (tid == 0 && n4 > 0 && !failed) {  // Q scale factors go to TMEM once
-    for (int i = 0; i < D / 64; ++i)
-      tc::tmem_cp_sf(tmem + COL_SFQ + 4 * i,
-                     tc::smem_desc(tc::smem_u32(smem + sm.q[0] + kSlots * D / 2 + i * kSfAtomBytes), 128, 128));
-  }
-  __syncthreads();
-
-  for (int i = 0; i < L && !s_abort; ++i) {
-    const int tier = tier_of_step(i);
-    const int b = min((int)ids[i], R - 1);
-    const uint32_t kvs = tc::smem_u32(smem + sm.kv[i & 1]);
-
-    // ------------------------------------------------------------ S = Q K^T (one thread issues)
-    if (tid == 0) {
-      if (!wait_or_abort(&bar_full[i & 1], (i >> 1) & 1, &s_abort)) { s_abort = 1; }
-      else {
-        tc::fence_after_sync();
-        const uint32_t qs = tc::smem_u32(smem + sm.q[tier]);
-        if (tier == 2) {
-          for (int ks = 0; ks < D / 16; ++ks)
-            tc::mma_f16(tmem + COL_S, tc::smem_desc(qs + ks * 2048, 1024, 128),
-                        tc::smem_desc(kvs + ks * 2048, 1024, 128), tc::idesc_bf16(64), ks > 0);
-        } else if (tier == 1) {
-          for (int ks = 0; ks < D / 32; ++ks)
-            tc::mma_i8(tmem + COL_S, tc::smem_desc(qs + ks * 2048, 1024, 128),
-                       tc::smem_desc(kvs + ks * 2048, 1024, 128), tc::idesc_i8(64), ks > 0);
-        } else {
-          const uint32_t ksf = kvs + kSlots * D / 2;
-          for (int j = 0; j < D / 64; ++j)
-            tc::tmem_cp_sf(tmem + COL_SFK + 4 * j, tc::smem_desc(ksf + j * kSfAtomBytes, 128, 128));
-          const uint32_t vsf = ksf + (D / 64) * kSfAtomBytes + D * kSlots / 2;
-          tc::tmem_cp_sf(tmem + COL_SFV, tc::smem_desc(vsf, 128, 128));
-          for (int ks = 0; ks < D / 64; ++ks)
-            tc::mma_nvfp4(tmem + COL_S, tc::smem_desc(qs + ks * 2048, 1024, 128),
-                          tc::smem_desc(kvs + ks * 2048, 1024, 128), tc::idesc_nvfp4(64), ks > 0,
-                          tmem + COL_SFQ + 4 * ks, tmem + COL_SFK + 4 * ks);
+  // =========================================================================================== loader warps
+  if (warp >= kLoadWarp0) {
+    const int s = warp - kLoadWarp0;
+    const StreamInfo S = s ? st1 : st0;
+    uint8_t *win = smem + sm.win + s * (kWindow * 14);
+    uint16_t *w_ids = reinterpret_cast<uint16_t *>(win);
+    float *w_dk = reinterpret_cast<float *>(win + kWindow * 2);
+    unsigned long long *w_mask = reinterpret_cast<unsigned long long *>(win + kWindow * 6);
+    if (lane == 0 && S.L > 0) {
+      const int nn[3] = {S.n4, S.n48 - S.n4, S.L - S.n48};
+      uint32_t bytes = 0;
+      for (int t = 0; t < 3; ++t) if (nn[t] > 0) bytes += p.qrec_bytes[t];
+      tc::mbar_arrive_expect_tx(bar(s, B_Q), bytes);
+      for (int t = 0; t < 3; ++t)
+        if (nn[t] > 0)
+          tc::bulk_g2s(smem + sm.q[s][t], p.qrec[t] + ((size_t)bh * R + S.a) * p.qrec_bytes[t], p.qrec_bytes[t],
+                       bar(s, B_Q));
+    }
+    int kk = 0, vv = 0, kround = 0, vround = 0;  // ring positions and how often each ring has wrapped
+    const size_t head_blocks = (size_t)bh * R;
+    for (int i = 0; i < S.L && !*abortp; ++i) {
+      const int j = i & (kWindow - 1);
+      if (j == 0) {  // stage the next window of list entries (ids, INT8 key scales, valid masks)
+        __syncwarp();
+        for (int jj = lane; jj < kWindow; jj += 32) {
+          const int idx = i + jj;
+          if (idx < S.L) {
+            int b = S.ids[idx];
+            if (b >= R) { atomicExch(p.status, kDevBadList); b = 0; }
+            w_ids[jj] = (uint16_t)b;
+            w_dk[jj] = S.tier(idx) == 1 ? p.dk8[head_blocks + b] : 0.f;
+            w_mask[jj] = block_valid_mask(p, b);
+          }
         }
-        tc::mma_commit(bar_s);
+        __syncwarp();
+      }
+      if (lane == 0) {
+        const int t = S.tier(i);
+        const uint8_t *rec = p.kvrec[t] + (head_blocks + w_ids[j]) * p.kvrec_bytes[t];
+        // the step's mask and key scale enter the info ring before the data the softmax waits for is requested
+        uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
+        *reinterpret_cast<unsigned long long *>(info) = w_mask[j];
+        *reinterpret_cast<float *>(info + 8) = w_dk[j];
+        if (kround > 0 && !wait_or_abort(bar(s, B_KFREE + kk), (kround - 1) & 1, abortp)) break;
+        tc::mbar_arrive_expect_tx(bar(s, B_FULLK + kk), sm.kbytes[t]);
+        tc::bulk_g2s(smem + sm.kst[s][0] + kk * sm.kstage, rec, sm.kbytes[t], bar(s, B_FULLK + kk));
+        if (vround > 0 && !wait_or_abort(bar(s, B_VFREE + vv), (vround - 1) & 1, abortp)) break;
+        tc::mbar_arrive_expect_tx(bar(s, B_FULLV + vv), sm.vbytes[t]);
+        tc::bulk_g2s(smem + sm.vst[s][0] + vv * sm.vstage, rec + sm.kbytes[t], sm.vbytes[t], bar(s, B_FULLV + vv));
+        if (++kk == sm.nk) { kk = 0; ++kround; }
+        if (++vv == sm.nv) { vv = 0; ++vround; }
       }
     }
-    if (!wait_or_abort(bar_s, i & 1, &s_abort)) { s_abort = 1; }
-    tc::fence_after_sync();
+  }
+  // =========================================================================================== MMA warps
+  else if (warp >= kMmaWarp0) {
+    const int s = warp - kMmaWarp0;
+    const StreamInfo S = s ? st1 : st0;
+    if (lane == 0 && S.L > 0 && wait_or_abort(bar(s, B_Q), 0, abortp)) {
+      // operand descriptors, built once; inside the loop only the 16-byte-unit start address (low bits) moves
+      const uint64_t qd0 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t qd1 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][1]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t qd2 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][2]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t kd0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]), 1024, 128);
+      const uint64_t vd0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]), D * 16, 128);
+      const uint64_t ksf0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]) + kSlots * D / 2, 128, 128);
+      const uint64_t vsf0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]) + D * kSlots / 2, 128, 128);
+      const uint64_t pd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.p[s][0]), 1024, 128),
+                              tc::smem_desc(tc::smem_u32(smem + sm.p[s][1]), 1024, 128)};
+      const uint64_t sfpd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][0]), 128, 128),
+                                tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][1]), 128, 128)};
+      const uint32_t kstep = sm.kstage >> 4, vstep = sm.vstage >> 4;
+      const uint32_t t_sfq = tmem + col_sfq(s), t_sfk = tmem + col_sfk(s), t_sfv = tmem + col_sfv(s),
+                     t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
+      if (S.n4 > 0) {  // Q scale factors go to TMEM once; the record carries them for rows 0..63 and again for rows
+                       // 64..127, so the same atom serves either stream
+#pragma unroll
+        for (int k = 0; k < D / 64; ++k)
+          tc::tmem_cp_sf(t_sfq + 4 * k, tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) + kSlots * D / 2 + k * kSfAtomBytes,
+                                                       128, 128));
+      }
+      int kk = 0, vv = 0;
+      uint32_t kpar = 0, vpar = 0;
+      for (int i = 0; i <= S.L; ++i) {
+        // ---- S(i) = Q K(i)^T
+        if (i < S.L) {
+          const int g = i & 1;
+          if (!wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp)) break;
+          if (!wait_or_abort(bar(s, B_SFREE + g), ((i >> 1) & 1) ^ 1, abortp)) break;
+          tc::fence_after_sync();
+          const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
+          const uint32_t d_s = tmem + col_s(s, g);
+          if (i >= S.n48) {
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
+          } else if (i >= S.n4) {
+#pragma unroll
+            for (int ks = 0; ks < D / 32; ++ks)
+              tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
+          } else {
+            const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
+#pragma unroll
+            for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
+#pragma unroll
+            for (int ks = 0; ks < D / 64; ++ks)
+              tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks,
+                            t_sfk + 4 * ks);
+          }
+          tc::mma_commit(bar(s, B_SREADY + g));
+          tc::mma_commit(bar(s, B_KFREE + kk));
+          if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
+        }
+        // ---- O^T += V(i-1)^T P(i-1)^T
+        if (i >= 1) {
+          const int j = i - 1, g = j & 1;
+          if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
+          if (!wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp)) break;
+          if (!wait_or_abort(bar(s, B_OCORR + g), (j >> 1) & 1, abortp)) break;
+          tc::fence_after_sync();
+          const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
+          const uint32_t acc = j > 0;
+          if (j >= S.n48) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
+          } else if (j >= S.n4) {
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks)
+              tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
+          } else {
+            tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
+            tc::tmem_cp_sf(t_sfp, sfpd[g]);
+            tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
+          }
+          tc::mma_commit(bar(s, B_PVDONE + g));
+          tc::mma_commit(bar(s, B_VFREE + vv));
+          if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
+        }
+      }
+    }
+  }
+  // =========================================================================================== softmax warps
+  else if (warp < kSoftmaxWarps) {
+    const int s = (warp & 3) >> 1, half = warp >> 2;
+    const int r = (warp & 1) * 32 + lane;  // query row inside the stream's block
+    const StreamInfo S = s ? st1 : st0;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const float gqk = p.gscale[bh * 4 + 0] * p.gscale[bh * 4 + 1] * p.scale * kLog2e;
+    const float dq8s = (S.a >= 0 && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
+    const float c16 = p.scale * kLog2e;
+    float h2 = -INFINITY, ell = 0.f;  // log2-domain running maximum; partial denominator over this thread's columns
 
-    // ------------------------------------------------------------ online softmax, one thread per query row
-    if (tid < kSlots && !s_abort) {
-      uint32_t raw[64];
+    for (int i = 0; i < S.L; ++i) {
+      const int g = i & 1, tier = S.tier(i);
+      if (!wait_or_abort(bar(s, B_SREADY + g), (i >> 1) & 1, abortp)) break;
+      tc::fence_after_sync();
+      uint32_t raw[32];
+      {
+        uint32_t a0[16], a1[16];
+        tc::tmem_ld16(tmem + lane_addr + col_s(s, g) + half * 32, a0);
+        tc::tmem_ld16(tmem + lane_addr + col_s(s, g) + half * 32 + 16, a1);
+        tc::wait_ld();
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t part[16];
-        tc::tmem_ld16(tmem + lane_base + COL_S + 16 * c, part);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) raw[16 * c + j] = part[j];
+        for (int j = 0; j < 16; ++j) { raw[j] = a0[j]; raw[16 + j] = a1[j]; }
       }
-      tc::wait_ld();
-      const unsigned long long kmask = block_valid_mask(p, b);
+      tc::fence_before_sync();
+      tc::mbar_arrive(bar(s, B_SFREE + g));
+
+      const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
+      const uint32_t kmask = *reinterpret_cast<const uint32_t *>(info + half * 4);
       float coef;
-      if (tier == 2) coef = p.scale * kLog2e;
-      else if (tier == 1) coef = dq8 * p.dk8[(size_t)bh * R + b] * p.scale * kLog2e;
-      else coef = gq * gk * p.scale * kLog2e;
-      float t[64];
-      float mloc = -INFINITY;
+      if (tier == 2) coef = c16;
+      else if (tier == 1) coef = dq8s * *reinterpret_cast<const float *>(info + 8);
+      else coef = gqk;
+
+      // scores as floats; int32 accumulators become floats exactly through a magic-number add and subtract
+      // (|S| < 2^22), two full-rate operations instead of a conversion on the special-function unit
+      float v[32];
+      if (tier == 1) {
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        const float sv = tier == 1 ? (float)(int)raw[j] : __uint_as_float(raw[j]);
-        t[j] = ((kmask >> j) & 1ull) ? sv * coef : -INFINITY;
-        mloc = fmaxf(mloc, t[j]);
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j] + 0x4B400000u) - 12582912.0f;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
       }
-      const float m_new = fmaxf(h2, mloc);
+      if (kmask != 0xffffffffu) {  // ragged edge tile: padding keys take no part (weight 0, outside every maximum)
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = ((kmask >> j) & 1u) ? v[j] : -INFINITY;
+      }
+      // maxima of the two 16-key groups, then of the 32 columns
+      float g0 = v[0], g1 = v[16];
+#pragma unroll
+      for (int j = 1; j < 16; ++j) { g0 = fmaxf(g0, v[j]); g1 = fmaxf(g1, v[16 + j]); }
+      const float pmax = fmaxf(g0, g1) * coef;  // log2 domain
+      s_xmax[((s * 2 + g) * 2 + half) * 64 + r] = pmax;
+      tc::mbar_arrive(bar(s, B_XREADY + g));
+      if (!wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp)) break;
+      const float other = s_xmax[((s * 2 + g) * 2 + (half ^ 1)) * 64 + r];
+      const float m_new = fmaxf(h2, fmaxf(pmax, other));
       const float factor = ex2(h2 - m_new);  // 0 on the first block (h2 = -inf)
-      s_factor[tid] = factor;
-      s_changed[tid] = (m_new != h2) ? 1 : 0;
+      if (half == 0) {
+        s_factor[(s * 2 + g) * 64 + r] = factor;
+        const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h2);
+        if (lane == 0) s_chg[(s * 2 + g) * 2 + (warp & 1)] = moved;
+        tc::mbar_arrive(bar(s, B_FREADY + g));
+      }
       ell *= factor;
       h2 = m_new;
-      uint8_t *prow = smem + sm.p + tid * 16;
+      // the P buffer of this parity was last read by PV(i-2)
+      if (i >= 2 && !wait_or_abort(bar(s, B_PVDONE + g), ((i >> 1) - 1) & 1, abortp)) break;
+
+      uint8_t *prow = smem + sm.p[s][g] + r * 16;
       if (tier == 2) {
+        const float bias = -m_new;
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < 4; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float w0 = ex2(t[c * 8 + 2 * j] - m_new), w1 = ex2(t[c * 8 + 2 * j + 1] - m_new);
+            const float w0 = ex2(fmaf(v[c * 8 + 2 * j], coef, bias)), w1 = ex2(fmaf(v[c * 8 + 2 * j + 1], coef, bias));
             sum += w0 + w1;
             w4[j] = pack_bf16x2(w0, w1);
           }
-          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + (half * 4 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         ell += sum;
       } else if (tier == 1) {
+        const float bias = kOffsetP8 - m_new;
         float sum = 0.f;
-        const float shift = kOffsetP8 - m_new;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t w4[4] = {0, 0, 0, 0};
+        for (int c = 0; c < 2; ++c) {
+          uint32_t w4[4];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float w0 = ex2(t[c * 16 + 2 * j] + shift), w1 = ex2(t[c * 16 + 2 * j + 1] + shift);
-            sum += w0 + w1;
-            w4[j >> 1] |= pack_e4m3x2(w0, w1) << (16 * (j & 1));
+          for (int j = 0; j < 4; ++j) {
+            const float w0 = ex2(fmaf(v[c * 16 + 4 * j + 0], coef, bias)), w1 = ex2(fmaf(v[c * 16 + 4 * j + 1], coef, bias));
+            const float w2 = ex2(fmaf(v[c * 16 + 4 * j + 2], coef, bias)), w3 = ex2(fmaf(v[c * 16 + 4 * j + 3], coef, bias));
+            sum += (w0 + w1) + (w2 + w3);
+            w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
           }
-          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + (half * 2 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
-        ell += kEtaP8 * sum;  // the denominator accumulates the amplified fp32 weights; eta restores the unit
+        ell += kEtaP8 * sum;  // the denominator sums the amplified fp32 weights; eta restores the unit
       } else {
-        float sum = 0.f;
-        uint32_t sfword = 0;
+        uint32_t w4[4];
+        uint32_t sfhalf = 0;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          float w[16];
-          float gm = 0.f;
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            w[j] = ex2(t[g * 16 + j] - m_new);
-            sum += w[j];
-            gm = fmaxf(gm, w[j]);
-          }
-          const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gm), 0.f) & 0xffu;
+        for (int gi = 0; gi < 2; ++gi) {
+          // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent
+          const float gw = ex2(fmaf(gi ? g1 : g0, coef, -m_new));
+          const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gw), 0.f) & 0xffu;
           const float sigma = decode_e4m3(sc);
-          sfword |= sc << (8 * g);
-          uint32_t w2[2] = {0, 0};
-          if (sigma > 0.f) {
-            const float inv = __fdiv_rn(2688.0f, sigma);
+          sfhalf |= sc << (8 * gi);
+          const bool live = sigma > 0.f;
+          const float bias = (live ? lg2(__fdiv_rn(2688.0f, sigma)) : 0.f) - m_new;
+          float sum = 0.f;
+          uint32_t c0 = 0, c1 = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) w2[j >> 2] |= pack_e2m1x2(w[2 * j] * inv, w[2 * j + 1] * inv) << (8 * (j & 3));
+          for (int j = 0; j < 4; ++j) {
+            const float u0 = ex2(fmaf(v[gi * 16 + 4 * j + 0], coef, bias)), u1 = ex2(fmaf(v[gi * 16 + 4 * j + 1], coef, bias));
+            const float u2 = ex2(fmaf(v[gi * 16 + 4 * j + 2], coef, bias)), u3 = ex2(fmaf(v[gi * 16 + 4 * j + 3], coef, bias));
+            sum += (u0 + u1) + (u2 + u3);
+            const uint32_t pk = pack_e2m1x4(u0, u1, u2, u3);
+            if (j < 2) c0 |= pk << (16 * j); else c1 |= pk << (16 * (j - 2));
           }
-          // 16 keys = 8 bytes: chunk g/2 (32 keys per 16-byte chunk), half g&1
-          *reinterpret_cast<uint2 *>(prow + (g >> 1) * 1024 + (g & 1) * 8) = make_uint2(w2[0], w2[1]);
+          w4[2 * gi] = live ? c0 : 0u;
+          w4[2 * gi + 1] = live ? c1 : 0u;
+          ell += sum * (live ? sigma * (1.0f / 2688.0f) : 1.0f);
         }
-        *reinterpret_cast<uint32_t *>(smem + sm.sfp + (tid & 31) * 16 + (tid >> 5) * 4) = sfword;
-        ell += sum;
+        *reinterpret_cast<uint4 *>(prow + half * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        *reinterpret_cast<uint16_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4 + half * 2) = (uint16_t)sfhalf;
       }
       tc::fence_async_smem();
+      tc::mbar_arrive(bar(s, B_PREADY + g));
     }
-    tc::fence_before_sync();
-    __syncthreads();
-    tc::fence_after_sync();
-    if (s_abort) break;
-
-    // ------------------------------------------------------------ correct the accumulator (all 128 lanes)
-    if (i > 0) {
-      float lane_factor = 1.0f;
-      const bool tier_switch = tier != prev_tier;
-      if (tier_switch && tid < D) {
-        const float un = unit_of(tier), up = unit_of(prev_tier);
-        lane_factor = un > 0.f ? __fdiv_rn(up, un) : 0.f;
-      }
-#pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        const unsigned long long ch = *reinterpret_cast<const unsigned long long *>(s_changed + c * 8);
-        if (ch == 0ull && !tier_switch) continue;
-        uint32_t o[8];
-        tc::tmem_ld8(tmem + lane_base + COL_O + c * 8, o);
-        tc::wait_ld();
-#pragma unroll
-        for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * (s_factor[c * 8 + j] * lane_factor));
-        tc::tmem_st8(tmem + lane_base + COL_O + c * 8, o);
-      }
-      tc::wait_st();
+    if (S.L > 0) {
+      s_ell[(s * 2 + half) * 64 + r] = ell;
+      tc::mbar_arrive(bar(s, B_ELL));
     }
-    prev_tier = tier;
-    tc::fence_before_sync();
-    __syncthreads();
-
-    // ------------------------------------------------------------ O^T += V^T P^T (one thread issues)
-    if (tid == 0) {
-      tc::fence_after_sync();
-      const uint32_t ps = tc::smem_u32(smem + sm.p);
-      if (tier == 2) {
-        const uint32_t vs = kvs + kSlots * D * 2;
-        for (int ks = 0; ks < 4; ++ks)
-          tc::mma_f16(tmem + COL_O, tc::smem_desc(vs + ks * 2 * D * 16, D * 16, 128),
-                      tc::smem_desc(ps + ks * 2048, 1024, 128), tc::idesc_bf16(64), (i > 0) || (ks > 0));
-      } else if (tier == 1) {
-        const uint32_t vs = kvs + kSlots * D;
-        for (int ks = 0; ks < 2; ++ks)
-          tc::mma_f8f6f4(tmem + COL_O, tc::smem_desc(vs + ks * 2 * D * 16, D * 16, 128),
-                         tc::smem_desc(ps + ks * 2048, 1024, 128), tc::idesc_e4m3(64), (i > 0) || (ks > 0));
-      } else {
-        const uint32_t vs = kvs + kSlots * D / 2 + (D / 64) * kSfAtomBytes;
-        tc::tmem_cp_sf(tmem + COL_SFP, tc::smem_desc(tc::smem_u32(smem + sm.sfp), 128, 128));
-        tc::mma_nvfp4(tmem + COL_O, tc::smem_desc(vs, D * 16, 128), tc::smem_desc(ps, 1024, 128),
-                      tc::idesc_nvfp4(64), i > 0, tmem + COL_SFV, tmem + COL_SFP);
-      }
-      tc::mma_commit(bar_o);
-    }
-    if (!wait_or_abort(bar_o, i & 1, &s_abort)) { s_abort = 1; }
-    tc::fence_after_sync();
-    __syncthreads();
-    if (tid == 0 && i + 2 < L && !s_abort) issue_kv(i + 2);
   }
-
-  if (s_abort) {
-    if (tid == 0) {
-      atomicExch(p.status, kDevTimeout);
-      // let any copy still in flight land before the shared memory goes away
-      tc::mbar_wait(&bar_full[0], 0, 1u << 16);
-      tc::mbar_wait(&bar_full[1], 0, 1u << 16);
-    }
-  } else {
-    // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
-    if (tid < kSlots) s_inv_l[tid] = ell > 0.f ? __fdiv_rn(1.0f, ell) : 0.f;
-    __syncthreads();
-    uint16_t *stage = reinterpret_cast<uint16_t *>(smem + sm.kv[0]);  // [64][D] bf16
-    const float unit = tid < D ? unit_of(prev_tier) : 0.f;
-#pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
-      uint32_t o[8];
-      tc::tmem_ld8(tmem + lane_base + COL_O + c * 8, o);
-      tc::wait_ld();
-      if (tid < D) {
+  // =========================================================================================== correction warps
+  else {
+    const int cw = warp - kSoftmaxWarps;       // lane quarter
+    const int ch = cw * 32 + lane;             // channel (TMEM lane)
+    const uint32_t lane_addr = (uint32_t)(cw * 32) << 16;
+    const float gv = p.gscale[bh * 4 + 2];
+    const float dv8 = (p.tier_active[1] && ch < D) ? p.dv8[(size_t)bh * D + ch] : 0.f;
+    auto unit_of = [&](int t) -> float {  // common units per accumulator unit, for this thread's channel
+      return t == 0 ? __fdiv_rn(gv, 2688.0f) : (t == 1 ? kEtaP8 * dv8 : 1.0f);
+    };
+    const int Lmax = max(st0.L, st1.L);
+    bool dead = false;
+    for (int i = 0; i < Lmax && !dead; ++i) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float val = __uint_as_float(o[j]) * unit * s_inv_l[c * 8 + j];
-          stage[(c * 8 + j) * D + tid] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
+      for (int s = 0; s < 2; ++s) {
+        const StreamInfo &S = s ? st1 : st0;
+        if (i >= S.L || dead) continue;
+        const int g = i & 1;
+        if (!wait_or_abort(bar(s, B_FREADY + g), (i >> 1) & 1, abortp)) { dead = true; continue; }
+        if (i > 0) {
+          const int tier = S.tier(i);
+          const bool tier_switch = (i == S.n4) || (i == S.n48);
+          const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * 2 + g) * 2);
+          if ((moved.x | moved.y) != 0u || tier_switch) {
+            if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp)) { dead = true; continue; }
+            tc::fence_after_sync();
+            float lane_factor = 1.0f;
+            if (tier_switch && ch < D) {
+              const float un = unit_of(tier), up = unit_of(S.tier(i - 1));
+              lane_factor = un > 0.f ? __fdiv_rn(up, un) : 0.f;
+            }
+            const float *fac = s_factor + (s * 2 + g) * 64;
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+              const uint32_t m8 = ((c < 4 ? moved.x : moved.y) >> ((c & 3) * 8)) & 0xffu;
+              if (m8 == 0u && !tier_switch) continue;
+              uint32_t o[8];
+              tc::tmem_ld8(tmem + lane_addr + col_o(s) + c * 8, o);
+              tc::wait_ld();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * (fac[c * 8 + j] * lane_factor));
+              tc::tmem_st8(tmem + lane_addr + col_o(s) + c * 8, o);
+            }
+            tc::wait_st();
+            tc::fence_before_sync();
+          }
+        }
+        tc::mbar_arrive(bar(s, B_OCORR + g));
+      }
+    }
+    // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const StreamInfo &S = s ? st1 : st0;
+      if (S.a < 0) continue;
+      const unsigned long long qmask = block_valid_mask(p, S.a);
+      uint16_t *stage = reinterpret_cast<uint16_t *>(smem + sm.kst[s][0]);  // [64][D] bf16 over the K ring
+      bool ok = S.L > 0 && !*abortp;
+      if (ok) ok = wait_or_abort(bar(s, B_ELL), 0, abortp);
+      if (ok) ok = wait_or_abort(bar(s, B_PVDONE + ((S.L - 1) & 1)), ((S.L - 1) >> 1) & 1, abortp);
+      if (ok) {
+        tc::fence_after_sync();
+        const float unit = ch < D ? unit_of(S.tier(S.L - 1)) : 0.f;
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          uint32_t o[8];
+          tc::tmem_ld8(tmem + lane_addr + col_o(s) + c * 8, o);
+          tc::wait_ld();
+          if (ch < D) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int qr = c * 8 + j;
+              const float l = s_ell[(s * 2 + 0) * 64 + qr] + s_ell[(s * 2 + 1) * 64 + qr];
+              const float val = l > 0.f ? __uint_as_float(o[j]) * unit * __fdiv_rn(1.0f, l) : 0.f;
+              stage[qr * D + ch] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
+            }
+          }
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (S.L == 0) {
+        store_zero_rows(S.a, tid - kSoftmaxWarps * 32, kCorrWarps * 32);
+      } else if (ok) {
+        for (int idx = tid - kSoftmaxWarps * 32; idx < kSlots * (D / 8); idx += kCorrWarps * 32) {
+          const int j = idx / (D / 8), c8 = idx % (D / 8);
+          if ((qmask >> j) & 1ull)
+            *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, S.a, j) * D + c8 * 8) =
+                *reinterpret_cast<const uint4 *>(stage + j * D + c8 * 8);
         }
       }
     }
-    __syncthreads();
-    for (int idx = tid; idx < kSlots * (D / 8); idx += NT) {
-      const int j = idx / (D / 8), c8 = idx % (D / 8);
-      if ((qmask >> j) & 1ull)
-        *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, a, j) * D + c8 * 8) =
-            *reinterpret_cast<const uint4 *>(stage + j * D + c8 * 8);
-    }
   }
+
   tc::fence_before_sync();
   __syncthreads();
+  if (s_abort && tid == 0) {
+    atomicExch(p.status, kDevTimeout);
+    atomicCAS(p.status + 1, 0, s_abort - 1 - (int)(tc::smem_u32(bars) & 0xffff));  // byte offset of the stuck barrier
+  }
   if (warp == 0) tc::tmem_dealloc(tmem, kTmemCols);
 }
 
@@ -430,7 +660,7 @@ __global__ void __launch_bounds__(NT) attention_kernel(Params p, SmemMap sm, __n
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches) {
   const SmemMap sm = make_smem_map(p);
   cudaError_t e;
-  const int grid = p.BH * p.R;
+  const int grid = p.BH * ((p.R + 1) / 2);
   if (p.d == 128) {
     e = cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
     if (e != cudaSuccess) return e;

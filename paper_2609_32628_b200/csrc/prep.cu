@@ -192,7 +192,10 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
           const uint32_t sc = nvfp4_group(x, g, pk);
           w[2 * h] = pk[0]; w[2 * h + 1] = pk[1];
           const int grp = kc * 2 + h;  // 16-channel group index; 4 groups per atom
-          sf_img[(grp >> 2) * kSfAtomBytes + (r & 31) * 16 + (r >> 5) * 4 + (grp & 3)] = (uint8_t)sc;
+          // rows 0..63 and, duplicated, rows 64..127: the attention kernel places a block's queries in either half
+          uint8_t *sfp = sf_img + (grp >> 2) * kSfAtomBytes + (r & 31) * 16 + (r >> 5) * 4 + (grp & 3);
+          sfp[0] = (uint8_t)sc;
+          sfp[8] = (uint8_t)sc;
         }
         *reinterpret_cast<uint4 *>(dst + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
