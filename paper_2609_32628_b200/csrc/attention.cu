@@ -170,18 +170,35 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
 // (the flag then holds 1 + the shared-memory offset of the barrier that was never completed, for diagnosis)
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
   if (tc::mbar_try_wait(bar, parity)) return true;
-  // The hand-offs between roles are on the critical path of every step, so the wait polls without sleeping (a
-  // sleep costs far more than a hand-off); the bound is on elapsed clock cycles.
+  // Waiting warps share their scheduler with the warps doing the softmax arithmetic, so they must not spin: each
+  // try suspends in hardware until the phase completes (or 20 us pass).  The bound is on elapsed clock cycles.
   const long long t0 = clock64();
-  for (uint32_t i = 1;; ++i) {
-    if (tc::mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > 400000000ll) break;  // about 0.2 s
-    }
+  for (;;) {
+    if (tc::mbar_try_wait_suspend(bar, parity, 20000u)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > 400000000ll) break;  // about 0.2 s
   }
   atomicCAS(const_cast<int *>(abort_flag), 0, 1 + (int)(tc::smem_u32(bar) & 0xffff));
   return false;
+}
+
+#ifdef DA2_PROF
+// Profiling build only: cycles spent in each wait site of one CTA, accumulated into the status words.
+#define PROF_WAIT(site, call) ([&]() { const long long t_ = clock64(); const bool ok_ = (call); \
+                                       prof_acc[site] += clock64() - t_; return ok_; }())
+#define PROF_T(var) const long long var = clock64()
+#define PROF_ADD(site, a, b) prof_acc[site] += (b) - (a)
+#else
+#define PROF_WAIT(site, call) (call)
+#define PROF_T(var)
+#define PROF_ADD(site, a, b)
+#endif
+
+// One arrival per warp: every lane's earlier writes are ordered before the elected lane's arrive by the warp barrier.
+// (A per-thread arrive is a shared-memory atomic per thread; hundreds of them per step dominate the step time.)
+__device__ __forceinline__ void warp_arrive(uint64_t *bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) tc::mbar_arrive(bar);
 }
 
 struct StreamInfo {
@@ -211,7 +228,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
   const int R = p.R, pairs = (R + 1) / 2;
   const int bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
   __nv_bfloat16 *out_head = out + (size_t)bh * p.N * D;
@@ -247,12 +265,12 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     for (int s = 0; s < 2; ++s) {
       for (int g = 0; g < 2; ++g) {
         tc::mbar_init(bar(s, B_SREADY + g), 1);
-        tc::mbar_init(bar(s, B_SFREE + g), 128);
-        tc::mbar_init(bar(s, B_PREADY + g), 128);
-        tc::mbar_init(bar(s, B_FREADY + g), 64);
-        tc::mbar_init(bar(s, B_XREADY + g), 128);
+        tc::mbar_init(bar(s, B_SFREE + g), 2);
+        tc::mbar_init(bar(s, B_PREADY + g), 2);
+        tc::mbar_init(bar(s, B_FREADY + g), 2);
+        tc::mbar_init(bar(s, B_XREADY + g), 2);
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
-        tc::mbar_init(bar(s, B_OCORR + g), 128);
+        tc::mbar_init(bar(s, B_OCORR + g), 4);
       }
       for (int g = 0; g < kMaxStages; ++g) {
         tc::mbar_init(bar(s, B_FULLK + g), 1);
@@ -260,7 +278,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         tc::mbar_init(bar(s, B_KFREE + g), 1);
         tc::mbar_init(bar(s, B_VFREE + g), 1);
       }
-      tc::mbar_init(bar(s, B_ELL), 128);
+      tc::mbar_init(bar(s, B_ELL), 4);
       tc::mbar_init(bar(s, B_Q), 1);
     }
     tc::fence_barrier_init();
@@ -271,6 +289,10 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   tc::fence_after_sync();
   const uint32_t tmem = s_tmem_base;
   volatile int *abortp = &s_abort;
+#ifdef DA2_PROF
+  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const long long prof_t0 = clock64();
+#endif
 
   // =========================================================================================== loader warps
   if (warp >= kLoadWarp0) {
@@ -315,10 +337,10 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
         *reinterpret_cast<unsigned long long *>(info) = w_mask[j];
         *reinterpret_cast<float *>(info + 8) = w_dk[j];
-        if (kround > 0 && !wait_or_abort(bar(s, B_KFREE + kk), (kround - 1) & 1, abortp)) break;
+        if (kround > 0 && !PROF_WAIT(0, wait_or_abort(bar(s, B_KFREE + kk), (kround - 1) & 1, abortp))) break;
         tc::mbar_arrive_expect_tx(bar(s, B_FULLK + kk), sm.kbytes[t]);
         tc::bulk_g2s(smem + sm.kst[s][0] + kk * sm.kstage, rec, sm.kbytes[t], bar(s, B_FULLK + kk));
-        if (vround > 0 && !wait_or_abort(bar(s, B_VFREE + vv), (vround - 1) & 1, abortp)) break;
+        if (vround > 0 && !PROF_WAIT(1, wait_or_abort(bar(s, B_VFREE + vv), (vround - 1) & 1, abortp))) break;
         tc::mbar_arrive_expect_tx(bar(s, B_FULLV + vv), sm.vbytes[t]);
         tc::bulk_g2s(smem + sm.vst[s][0] + vv * sm.vstage, rec + sm.kbytes[t], sm.vbytes[t], bar(s, B_FULLV + vv));
         if (++kk == sm.nk) { kk = 0; ++kround; }
@@ -328,9 +350,15 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   }
   // =========================================================================================== MMA warps
   else if (warp >= kMmaWarp0) {
+    // The whole warp runs this loop with warp-uniform control flow and values; only the tcgen05 instructions
+    // themselves are issued by one elected lane.  (Under a lane-0 branch every descriptor would have to be moved from
+    // vector to uniform registers before each issue, which costs more than the MMA itself.)
     const int s = warp - kMmaWarp0;
-    const StreamInfo S = s ? st1 : st0;
-    if (lane == 0 && S.L > 0 && wait_or_abort(bar(s, B_Q), 0, abortp)) {
+    StreamInfo S = s ? st1 : st0;
+    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
+    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
+    S.L = __shfl_sync(0xffffffffu, S.L, 0);
+    if (S.L > 0 && wait_or_abort(bar(s, B_Q), 0, abortp)) {
       // operand descriptors, built once; inside the loop only the 16-byte-unit start address (low bits) moves
       const uint64_t qd0 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) - (s ? 1024u : 0u), 1024, 128);
       const uint64_t qd1 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][1]) - (s ? 1024u : 0u), 1024, 128);
@@ -348,148 +376,189 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
                      t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
       if (S.n4 > 0) {  // Q scale factors go to TMEM once; the record carries them for rows 0..63 and again for rows
                        // 64..127, so the same atom serves either stream
+        if (tc::elect_one()) {
 #pragma unroll
-        for (int k = 0; k < D / 64; ++k)
-          tc::tmem_cp_sf(t_sfq + 4 * k, tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) + kSlots * D / 2 + k * kSfAtomBytes,
-                                                       128, 128));
+          for (int k = 0; k < D / 64; ++k)
+            tc::tmem_cp_sf(t_sfq + 4 * k, tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) + kSlots * D / 2 + k * kSfAtomBytes,
+                                                         128, 128));
+        }
       }
       int kk = 0, vv = 0;
       uint32_t kpar = 0, vpar = 0;
-      for (int i = 0; i <= S.L; ++i) {
-        // ---- S(i) = Q K(i)^T
-        if (i < S.L) {
-          const int g = i & 1;
-          if (!wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp)) break;
-          if (!wait_or_abort(bar(s, B_SFREE + g), ((i >> 1) & 1) ^ 1, abortp)) break;
-          tc::fence_after_sync();
-          const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
-          const uint32_t d_s = tmem + col_s(s, g);
-          if (i >= S.n48) {
+      bool alive = true;
+      // S(j) = Q K(j)^T
+      auto issue_qk = [&](int j) {
+        const int g = j & 1;
+        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp))) { alive = false; return; }
+        if (!PROF_WAIT(1, wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp))) { alive = false; return; }
+        tc::fence_after_sync();
+        PROF_T(mq0);
+        const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
+        const uint32_t d_s = tmem + col_s(s, g);
+        if (tc::elect_one()) {
+        if (j >= S.n48) {
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks)
-              tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
-          } else if (i >= S.n4) {
+          for (int ks = 0; ks < D / 16; ++ks) tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
+        } else if (j >= S.n4) {
 #pragma unroll
-            for (int ks = 0; ks < D / 32; ++ks)
-              tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
-          } else {
-            const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
+          for (int ks = 0; ks < D / 32; ++ks) tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
+        } else {
+          const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
 #pragma unroll
-            for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
+          for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
 #pragma unroll
-            for (int ks = 0; ks < D / 64; ++ks)
-              tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks,
-                            t_sfk + 4 * ks);
-          }
-          tc::mma_commit(bar(s, B_SREADY + g));
-          tc::mma_commit(bar(s, B_KFREE + kk));
-          if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
+          for (int ks = 0; ks < D / 64; ++ks)
+            tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks, t_sfk + 4 * ks);
         }
-        // ---- O^T += V(i-1)^T P(i-1)^T
-        if (i >= 1) {
-          const int j = i - 1, g = j & 1;
-          if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
-          if (!wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp)) break;
-          if (!wait_or_abort(bar(s, B_OCORR + g), (j >> 1) & 1, abortp)) break;
-          tc::fence_after_sync();
-          const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
-          const uint32_t acc = j > 0;
-          if (j >= S.n48) {
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
-          } else if (j >= S.n4) {
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks)
-              tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
-          } else {
-            tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
-            tc::tmem_cp_sf(t_sfp, sfpd[g]);
-            tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
-          }
-          tc::mma_commit(bar(s, B_PVDONE + g));
-          tc::mma_commit(bar(s, B_VFREE + vv));
-          if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
+        tc::mma_commit(bar(s, B_SREADY + g));
+        tc::mma_commit(bar(s, B_KFREE + kk));
         }
+        __syncwarp();
+        PROF_T(mq1);
+        PROF_ADD(5, mq0, mq1);
+        if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
+      };
+      // the score tiles are double buffered, so Q K^T runs two steps ahead of the accumulation
+      issue_qk(0);
+      if (alive && S.L > 1) issue_qk(1);
+      for (int j = 0; j < S.L && alive; ++j) {
+        if (j + 2 < S.L) { issue_qk(j + 2); if (!alive) break; }
+        // ---- O^T += V(j)^T P(j)^T
+        const int g = j & 1;
+        if (!PROF_WAIT(2, wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp))) break;
+        if (!PROF_WAIT(3, wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp))) break;
+        if (!PROF_WAIT(4, wait_or_abort(bar(s, B_OCORR + g), (j >> 1) & 1, abortp))) break;
+        tc::fence_after_sync();
+        PROF_T(mp0);
+        const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
+        const uint32_t acc = j > 0;
+        if (tc::elect_one()) {
+        if (j >= S.n48) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
+        } else if (j >= S.n4) {
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks)
+            tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
+        } else {
+          tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
+          tc::tmem_cp_sf(t_sfp, sfpd[g]);
+          tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
+        }
+        tc::mma_commit(bar(s, B_PVDONE + g));
+        tc::mma_commit(bar(s, B_VFREE + vv));
+        }
+        __syncwarp();
+        PROF_T(mp1);
+        PROF_ADD(6, mp0, mp1);
+        if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
       }
     }
   }
   // =========================================================================================== softmax warps
   else if (warp < kSoftmaxWarps) {
-    const int s = (warp & 3) >> 1, half = warp >> 2;
+    // The two softmax warps that share a scheduler (warp w and w+4) own the same 32 query rows and take ALTERNATE
+    // steps, one thread per full 64-key row: while one exponentiates and packs its step (special-function bound),
+    // the other fetches, masks and reduces the next one.  The only hand-off between them is the running maximum.
+    const int s = (warp & 3) >> 1, par = warp >> 2;
     const int r = (warp & 1) * 32 + lane;  // query row inside the stream's block
     const StreamInfo S = s ? st1 : st0;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const float gqk = p.gscale[bh * 4 + 0] * p.gscale[bh * 4 + 1] * p.scale * kLog2e;
     const float dq8s = (S.a >= 0 && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
     const float c16 = p.scale * kLog2e;
-    float h2 = -INFINITY, ell = 0.f;  // log2-domain running maximum; partial denominator over this thread's columns
+    float h_own = -INFINITY, ell = 0.f;  // log2-domain maximum after this warp's last step; its partial denominator
+    const int g = par;                   // buffers of this warp's step parity
+    float *my_h = s_xmax + ((s * 2 + g) * 2 + 0) * 64 + r;           // published running maximum of my steps
+    const float *other_h = s_xmax + ((s * 2 + (g ^ 1)) * 2 + 0) * 64 + r;
+    const uint32_t s_col = tmem + lane_addr + col_s(s, g);
+    uint8_t *prow = smem + sm.p[s][g] + r * 16;
 
-    for (int i = 0; i < S.L; ++i) {
-      const int g = i & 1, tier = S.tier(i);
-      if (!wait_or_abort(bar(s, B_SREADY + g), (i >> 1) & 1, abortp)) break;
+    for (int i = par; i < S.L; i += 2) {
+      const int tier = S.tier(i);
+      const uint32_t kp = (uint32_t)(i >> 1) & 1u;  // completion parity of this parity's k-th step
+      if (!PROF_WAIT(0, wait_or_abort(bar(s, B_SREADY + g), kp, abortp))) break;
       tc::fence_after_sync();
-      uint32_t raw[32];
+      PROF_T(pt0);
+      float v[64];
       {
-        uint32_t a0[16], a1[16];
-        tc::tmem_ld16(tmem + lane_addr + col_s(s, g) + half * 32, a0);
-        tc::tmem_ld16(tmem + lane_addr + col_s(s, g) + half * 32 + 16, a1);
+        uint32_t a0[16], a1[16], a2[16], a3[16];
+        tc::tmem_ld16(s_col, a0);
+        tc::tmem_ld16(s_col + 16, a1);
+        tc::tmem_ld16(s_col + 32, a2);
+        tc::tmem_ld16(s_col + 48, a3);
         tc::wait_ld();
+        // int32 accumulators become floats exactly through a magic-number add and subtract (|S| < 2^22): two
+        // full-rate operations instead of a conversion on the special-function unit
+        if (tier == 1) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { raw[j] = a0[j]; raw[16 + j] = a1[j]; }
+          for (int c = 0; c < 16; ++c) {
+            v[c] = __uint_as_float(a0[c] + 0x4B400000u) - 12582912.0f;
+            v[16 + c] = __uint_as_float(a1[c] + 0x4B400000u) - 12582912.0f;
+            v[32 + c] = __uint_as_float(a2[c] + 0x4B400000u) - 12582912.0f;
+            v[48 + c] = __uint_as_float(a3[c] + 0x4B400000u) - 12582912.0f;
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            v[c] = __uint_as_float(a0[c]); v[16 + c] = __uint_as_float(a1[c]);
+            v[32 + c] = __uint_as_float(a2[c]); v[48 + c] = __uint_as_float(a3[c]);
+          }
+        }
       }
+      PROF_T(pt1);
+      PROF_ADD(3, pt0, pt1);
       tc::fence_before_sync();
-      tc::mbar_arrive(bar(s, B_SFREE + g));
-
+      warp_arrive(bar(s, B_SFREE + g));
       const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
-      const uint32_t kmask = *reinterpret_cast<const uint32_t *>(info + half * 4);
+      const uint2 kmask = *reinterpret_cast<const uint2 *>(info);
       float coef;
       if (tier == 2) coef = c16;
       else if (tier == 1) coef = dq8s * *reinterpret_cast<const float *>(info + 8);
       else coef = gqk;
+      if ((kmask.x & kmask.y) != 0xffffffffu) {  // ragged edge tile: padding keys take no part
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          v[c] = ((kmask.x >> c) & 1u) ? v[c] : -INFINITY;
+          v[32 + c] = ((kmask.y >> c) & 1u) ? v[32 + c] : -INFINITY;
+        }
+      }
+      // maxima of the four 16-key groups (pairwise trees), then of the row
+      float gm[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float t8[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) t8[c] = fmaxf(v[q * 16 + c], v[q * 16 + 8 + c]);
+        gm[q] = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
+      }
+      const float pmax = fmaxf(fmaxf(gm[0], gm[1]), fmaxf(gm[2], gm[3])) * coef;  // log2 domain
+      PROF_T(pt2);
+      PROF_ADD(4, pt1, pt2);
+      // PV(i-2) done: this parity's P buffer is free and the correction warps are past step i-2
+      if (i >= 2 && !PROF_WAIT(1, wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp))) break;
+      // running maximum after step i-1, published by the other warp
+      float h_prev = -INFINITY;
+      if (i > 0) {
+        if (!PROF_WAIT(2, wait_or_abort(bar(s, B_XREADY + (g ^ 1)), (uint32_t)((i - 1) >> 1) & 1u, abortp))) break;
+        h_prev = *other_h;
+      }
+      const float m_new = fmaxf(h_prev, pmax);
+      *my_h = m_new;
+      s_factor[(s * 2 + g) * 64 + r] = ex2(h_prev - m_new);  // 0 on the first block (h_prev = -inf)
+      const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h_prev);
+      if (lane == 0) s_chg[(s * 2 + g) * 2 + (warp & 1)] = moved;
+      warp_arrive(bar(s, B_XREADY + g));  // the other warp's next step and the correction warps wait on this
+      ell *= ex2(h_own - m_new);
+      h_own = m_new;
 
-      // scores as floats; int32 accumulators become floats exactly through a magic-number add and subtract
-      // (|S| < 2^22), two full-rate operations instead of a conversion on the special-function unit
-      float v[32];
-      if (tier == 1) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j] + 0x4B400000u) - 12582912.0f;
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
-      }
-      if (kmask != 0xffffffffu) {  // ragged edge tile: padding keys take no part (weight 0, outside every maximum)
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = ((kmask >> j) & 1u) ? v[j] : -INFINITY;
-      }
-      // maxima of the two 16-key groups, then of the 32 columns
-      float g0 = v[0], g1 = v[16];
-#pragma unroll
-      for (int j = 1; j < 16; ++j) { g0 = fmaxf(g0, v[j]); g1 = fmaxf(g1, v[16 + j]); }
-      const float pmax = fmaxf(g0, g1) * coef;  // log2 domain
-      s_xmax[((s * 2 + g) * 2 + half) * 64 + r] = pmax;
-      tc::mbar_arrive(bar(s, B_XREADY + g));
-      if (!wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp)) break;
-      const float other = s_xmax[((s * 2 + g) * 2 + (half ^ 1)) * 64 + r];
-      const float m_new = fmaxf(h2, fmaxf(pmax, other));
-      const float factor = ex2(h2 - m_new);  // 0 on the first block (h2 = -inf)
-      if (half == 0) {
-        s_factor[(s * 2 + g) * 64 + r] = factor;
-        const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h2);
-        if (lane == 0) s_chg[(s * 2 + g) * 2 + (warp & 1)] = moved;
-        tc::mbar_arrive(bar(s, B_FREADY + g));
-      }
-      ell *= factor;
-      h2 = m_new;
-      // the P buffer of this parity was last read by PV(i-2)
-      if (i >= 2 && !wait_or_abort(bar(s, B_PVDONE + g), ((i >> 1) - 1) & 1, abortp)) break;
-
-      uint8_t *prow = smem + sm.p[s][g] + r * 16;
+      PROF_T(pt3);
       if (tier == 2) {
         const float bias = -m_new;
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 8; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -497,14 +566,14 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             sum += w0 + w1;
             w4[j] = pack_bf16x2(w0, w1);
           }
-          *reinterpret_cast<uint4 *>(prow + (half * 4 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         ell += sum;
       } else if (tier == 1) {
         const float bias = kOffsetP8 - m_new;
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < 4; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -513,19 +582,18 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             sum += (w0 + w1) + (w2 + w3);
             w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
           }
-          *reinterpret_cast<uint4 *>(prow + (half * 2 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         ell += kEtaP8 * sum;  // the denominator sums the amplified fp32 weights; eta restores the unit
       } else {
-        uint32_t w4[4];
-        uint32_t sfhalf = 0;
+        uint32_t sfword = 0;
 #pragma unroll
-        for (int gi = 0; gi < 2; ++gi) {
+        for (int gi = 0; gi < 4; ++gi) {
           // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent
-          const float gw = ex2(fmaf(gi ? g1 : g0, coef, -m_new));
+          const float gw = ex2(fmaf(gm[gi], coef, -m_new));
           const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gw), 0.f) & 0xffu;
           const float sigma = decode_e4m3(sc);
-          sfhalf |= sc << (8 * gi);
+          sfword |= sc << (8 * gi);
           const bool live = sigma > 0.f;
           const float bias = (live ? lg2(__fdiv_rn(2688.0f, sigma)) : 0.f) - m_new;
           float sum = 0.f;
@@ -538,19 +606,23 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             const uint32_t pk = pack_e2m1x4(u0, u1, u2, u3);
             if (j < 2) c0 |= pk << (16 * j); else c1 |= pk << (16 * (j - 2));
           }
-          w4[2 * gi] = live ? c0 : 0u;
-          w4[2 * gi + 1] = live ? c1 : 0u;
+          // 16 keys = 8 bytes: chunk gi/2 (32 keys per 16-byte chunk), half gi&1
+          *reinterpret_cast<uint2 *>(prow + (gi >> 1) * 1024 + (gi & 1) * 8) = make_uint2(live ? c0 : 0u, live ? c1 : 0u);
           ell += sum * (live ? sigma * (1.0f / 2688.0f) : 1.0f);
         }
-        *reinterpret_cast<uint4 *>(prow + half * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-        *reinterpret_cast<uint16_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4 + half * 2) = (uint16_t)sfhalf;
+        *reinterpret_cast<uint32_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4) = sfword;
       }
+      PROF_T(pt4);
+      PROF_ADD(5, pt3, pt4);
       tc::fence_async_smem();
-      tc::mbar_arrive(bar(s, B_PREADY + g));
+      warp_arrive(bar(s, B_PREADY + g));
+      PROF_T(pt5);
+      PROF_ADD(6, pt4, pt5);
     }
     if (S.L > 0) {
-      s_ell[(s * 2 + half) * 64 + r] = ell;
-      tc::mbar_arrive(bar(s, B_ELL));
+      s_ell[(s * 2 + par) * 64 + r] = ell;
+      s_xmax[((s * 2 + par) * 2 + 1) * 64 + r] = h_own;  // reference of this partial denominator
+      warp_arrive(bar(s, B_ELL));
     }
   }
   // =========================================================================================== correction warps
@@ -571,13 +643,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         const StreamInfo &S = s ? st1 : st0;
         if (i >= S.L || dead) continue;
         const int g = i & 1;
-        if (!wait_or_abort(bar(s, B_FREADY + g), (i >> 1) & 1, abortp)) { dead = true; continue; }
+        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp))) { dead = true; continue; }
         if (i > 0) {
           const int tier = S.tier(i);
           const bool tier_switch = (i == S.n4) || (i == S.n48);
           const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * 2 + g) * 2);
           if ((moved.x | moved.y) != 0u || tier_switch) {
-            if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp)) { dead = true; continue; }
+            if (!PROF_WAIT(1, wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp))) { dead = true; continue; }
             tc::fence_after_sync();
             float lane_factor = 1.0f;
             if (tier_switch && ch < D) {
@@ -600,7 +672,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             tc::fence_before_sync();
           }
         }
-        tc::mbar_arrive(bar(s, B_OCORR + g));
+        warp_arrive(bar(s, B_OCORR + g));
       }
     }
     // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
@@ -625,7 +697,10 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const int qr = c * 8 + j;
-              const float l = s_ell[(s * 2 + 0) * 64 + qr] + s_ell[(s * 2 + 1) * 64 + qr];
+              // the two warps of a row kept partial denominators relative to their own last maximum
+              const float h0 = s_xmax[((s * 2 + 0) * 2 + 1) * 64 + qr], h1 = s_xmax[((s * 2 + 1) * 2 + 1) * 64 + qr];
+              const float hf = fmaxf(h0, h1);
+              const float l = s_ell[(s * 2 + 0) * 64 + qr] * ex2(h0 - hf) + s_ell[(s * 2 + 1) * 64 + qr] * ex2(h1 - hf);
               const float val = l > 0.f ? __uint_as_float(o[j]) * unit * __fdiv_rn(1.0f, l) : 0.f;
               stage[qr * D + ch] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
             }
@@ -646,6 +721,15 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     }
   }
 
+#ifdef DA2_PROF
+  if (blockIdx.x == gridDim.x / 2 && lane == 0) {
+    const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == 8 ? 2 : warp == 12 ? 3 : warp == 14 ? 4 : -1;
+    if (role >= 0) {
+      prof_acc[7] = clock64() - prof_t0;
+      for (int k = 0; k < 8; ++k) p.status[8 + role * 8 + k] = (int)(prof_acc[k] >> 4);  // units of 16 cycles
+    }
+  }
+#endif
   tc::fence_before_sync();
   __syncthreads();
   if (s_abort && tid == 0) {
