@@ -142,6 +142,42 @@ __device__ __forceinline__ float lg2(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// packed pairs of fp32 (two lanes per instruction on this architecture) and a three-input maximum
+__device__ __forceinline__ uint64_t f2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unf2(uint64_t x, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(x)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// maximum of 16 values in 8 instructions
+__device__ __forceinline__ float max16(const float *x) {
+  const float m0 = max3(x[0], x[1], x[2]), m1 = max3(x[3], x[4], x[5]), m2 = max3(x[6], x[7], x[8]);
+  const float m3 = max3(x[9], x[10], x[11]), m4 = max3(x[12], x[13], x[14]);
+  return fmaxf(max3(m0, m1, m2), max3(m3, m4, x[15]));
+}
+// exponentials of two scores: 2^(x*coef + bias) for a packed pair (one packed FMA, two ex2)
+__device__ __forceinline__ void exp_pair(float x0, float x1, uint64_t coef2, uint64_t bias2, float &w0, float &w1) {
+  float t0, t1;
+  unf2(fma2(f2(x0, x1), coef2, bias2), t0, t1);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w0) : "f"(t0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w1) : "f"(t1));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -492,12 +528,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         // int32 accumulators become floats exactly through a magic-number add and subtract (|S| < 2^22): two
         // full-rate operations instead of a conversion on the special-function unit
         if (tier == 1) {
+          const uint64_t moff = f2(-12582912.0f, -12582912.0f);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            v[c] = __uint_as_float(a0[c] + 0x4B400000u) - 12582912.0f;
-            v[16 + c] = __uint_as_float(a1[c] + 0x4B400000u) - 12582912.0f;
-            v[32 + c] = __uint_as_float(a2[c] + 0x4B400000u) - 12582912.0f;
-            v[48 + c] = __uint_as_float(a3[c] + 0x4B400000u) - 12582912.0f;
+          for (int c = 0; c < 16; c += 2) {
+            unf2(add2(f2(__uint_as_float(a0[c] + 0x4B400000u), __uint_as_float(a0[c + 1] + 0x4B400000u)), moff), v[c], v[c + 1]);
+            unf2(add2(f2(__uint_as_float(a1[c] + 0x4B400000u), __uint_as_float(a1[c + 1] + 0x4B400000u)), moff), v[16 + c], v[17 + c]);
+            unf2(add2(f2(__uint_as_float(a2[c] + 0x4B400000u), __uint_as_float(a2[c + 1] + 0x4B400000u)), moff), v[32 + c], v[33 + c]);
+            unf2(add2(f2(__uint_as_float(a3[c] + 0x4B400000u), __uint_as_float(a3[c + 1] + 0x4B400000u)), moff), v[48 + c], v[49 + c]);
           }
         } else {
 #pragma unroll
@@ -527,13 +564,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       // maxima of the four 16-key groups (pairwise trees), then of the row
       float gm[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float t8[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) t8[c] = fmaxf(v[q * 16 + c], v[q * 16 + 8 + c]);
-        gm[q] = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
-      }
-      const float pmax = fmaxf(fmaxf(gm[0], gm[1]), fmaxf(gm[2], gm[3])) * coef;  // log2 domain
+      for (int q = 0; q < 4; ++q) gm[q] = max16(v + q * 16);
+      const float pmax = fmaxf(max3(gm[0], gm[1], gm[2]), gm[3]) * coef;  // log2 domain
       PROF_T(pt2);
       PROF_ADD(4, pt1, pt2);
       // PV(i-2) done: this parity's P buffer is free and the correction warps are past step i-2
@@ -554,61 +586,75 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       h_own = m_new;
 
       PROF_T(pt3);
+      const uint64_t coef2 = f2(coef, coef);
       if (tier == 2) {
-        const float bias = -m_new;
-        float sum = 0.f;
+        const uint64_t bias2 = f2(-m_new, -m_new);
+        uint64_t sum2 = 0;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float w0 = ex2(fmaf(v[c * 8 + 2 * j], coef, bias)), w1 = ex2(fmaf(v[c * 8 + 2 * j + 1], coef, bias));
-            sum += w0 + w1;
+            float w0, w1;
+            exp_pair(v[c * 8 + 2 * j], v[c * 8 + 2 * j + 1], coef2, bias2, w0, w1);
+            sum2 = add2(sum2, f2(w0, w1));
             w4[j] = pack_bf16x2(w0, w1);
           }
           *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
-        ell += sum;
+        float s0, s1;
+        unf2(sum2, s0, s1);
+        ell += s0 + s1;
       } else if (tier == 1) {
-        const float bias = kOffsetP8 - m_new;
-        float sum = 0.f;
+        const uint64_t bias2 = f2(kOffsetP8 - m_new, kOffsetP8 - m_new);
+        uint64_t sum2 = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float w0 = ex2(fmaf(v[c * 16 + 4 * j + 0], coef, bias)), w1 = ex2(fmaf(v[c * 16 + 4 * j + 1], coef, bias));
-            const float w2 = ex2(fmaf(v[c * 16 + 4 * j + 2], coef, bias)), w3 = ex2(fmaf(v[c * 16 + 4 * j + 3], coef, bias));
-            sum += (w0 + w1) + (w2 + w3);
+            float w0, w1, w2, w3;
+            exp_pair(v[c * 16 + 4 * j + 0], v[c * 16 + 4 * j + 1], coef2, bias2, w0, w1);
+            exp_pair(v[c * 16 + 4 * j + 2], v[c * 16 + 4 * j + 3], coef2, bias2, w2, w3);
+            sum2 = add2(add2(sum2, f2(w0, w1)), f2(w2, w3));
             w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
           }
           *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
-        ell += kEtaP8 * sum;  // the denominator sums the amplified fp32 weights; eta restores the unit
+        float s0, s1;
+        unf2(sum2, s0, s1);
+        ell += kEtaP8 * (s0 + s1);  // the denominator sums the amplified fp32 weights; eta restores the unit
       } else {
         uint32_t sfword = 0;
 #pragma unroll
         for (int gi = 0; gi < 4; ++gi) {
-          // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent
+          // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent:
+          // sigma = E4M3(448 * max w); scaled weight u = w * 2688 / sigma = 2^(x - m + log2(2688) - log2(sigma))
           const float gw = ex2(fmaf(gm[gi], coef, -m_new));
           const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gw), 0.f) & 0xffu;
-          const float sigma = decode_e4m3(sc);
           sfword |= sc << (8 * gi);
-          const bool live = sigma > 0.f;
-          const float bias = (live ? lg2(__fdiv_rn(2688.0f, sigma)) : 0.f) - m_new;
-          float sum = 0.f;
+          // E4M3 code -> fp32: for normal codes the bit pattern is a shift and a re-bias; the 7 subnormal codes
+          // and zero (weights below 2^-15 of the row maximum) take the general conversion
+          const float sigma = sc >= 8u ? __uint_as_float((sc << 20) + 0x3C000000u) : decode_e4m3(sc);
+          const bool live = sc != 0u;
+          const float b = (live ? 11.392317422778762f - lg2(sigma) : 0.f) - m_new;  // log2(2688) = 11.3923...
+          const uint64_t bias2 = f2(b, b);
+          uint64_t sum2 = 0;
           uint32_t c0 = 0, c1 = 0;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float u0 = ex2(fmaf(v[gi * 16 + 4 * j + 0], coef, bias)), u1 = ex2(fmaf(v[gi * 16 + 4 * j + 1], coef, bias));
-            const float u2 = ex2(fmaf(v[gi * 16 + 4 * j + 2], coef, bias)), u3 = ex2(fmaf(v[gi * 16 + 4 * j + 3], coef, bias));
-            sum += (u0 + u1) + (u2 + u3);
+            float u0, u1, u2, u3;
+            exp_pair(v[gi * 16 + 4 * j + 0], v[gi * 16 + 4 * j + 1], coef2, bias2, u0, u1);
+            exp_pair(v[gi * 16 + 4 * j + 2], v[gi * 16 + 4 * j + 3], coef2, bias2, u2, u3);
+            sum2 = add2(add2(sum2, f2(u0, u1)), f2(u2, u3));
             const uint32_t pk = pack_e2m1x4(u0, u1, u2, u3);
             if (j < 2) c0 |= pk << (16 * j); else c1 |= pk << (16 * (j - 2));
           }
           // 16 keys = 8 bytes: chunk gi/2 (32 keys per 16-byte chunk), half gi&1
           *reinterpret_cast<uint2 *>(prow + (gi >> 1) * 1024 + (gi & 1) * 8) = make_uint2(live ? c0 : 0u, live ? c1 : 0u);
-          ell += sum * (live ? sigma * (1.0f / 2688.0f) : 1.0f);
+          float s0, s1;
+          unf2(sum2, s0, s1);
+          ell = fmaf(s0 + s1, live ? sigma * (1.0f / 2688.0f) : 1.0f, ell);
         }
         *reinterpret_cast<uint32_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4) = sfword;
       }
