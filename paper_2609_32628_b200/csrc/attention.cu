@@ -7,15 +7,16 @@
 // the accumulator only changes units (Eq. "precision-state-conversion"), and the output is normalised once.
 //
 // Mapping onto sm_100a
-//   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 512 threads in four roles:
+//   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 576 threads in five roles:
 //     warps 0-7   softmax: stream = (warp%4)/2, two threads per query row (32 of the 64 key columns each); they read
 //                 S from TMEM, keep h and a partial l, and write P~ (and its NVFP4 scale factors) to shared memory
 //     warps 8-11  correction + epilogue: rescale the accumulator columns of queries whose maximum moved, apply the
 //                 per-channel unit change at a segment boundary, and finally normalise, transpose and store
-//     warps 12,13 MMA issue, one thread per stream: S = Q K^T and O^T += V^T P~^T with tcgen05.mma, accumulators
-//                 in TMEM.  This thread's instruction count is on the critical path of every step, so its operand
+//     warps 12,13 S = Q K^T issue, one warp per stream (tcgen05.mma, accumulators in TMEM), two steps ahead
+//     warps 14,15 O^T += V^T P~^T issue, one warp per stream.  The issuing warps' instruction counts are on the
+//                 critical path of every step: their loops are warp-uniform (one elected lane issues), operand
 //                 descriptors are built once and only offset inside the loop
-//     warps 14,15 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings
+//     warps 16,17 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings
 //   S   = Q K^T   : M = 128, N = 64 keys, K = d.  The block-scaled instruction only exists at M = 128, so stream 0's
 //                   queries sit in rows 0..63 and stream 1's in rows 64..127 (its operand descriptor starts 1 KB
 //                   early); the other 64 rows of each product are don't-care.  S is double buffered.
@@ -40,9 +41,10 @@ namespace da2 {
 namespace {
 
 constexpr int kSoftmaxWarps = 8, kCorrWarps = 4;
-constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // warps 12, 13: MMA issue for stream 0, 1
-constexpr int kLoadWarp0 = kMmaWarp0 + 2;              // warps 14, 15: loader for stream 0, 1
-constexpr int NT = (kLoadWarp0 + 2) * 32;              // 512
+constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // warps 12, 13: Q K^T issue for stream 0, 1
+constexpr int kPvWarp0 = kMmaWarp0 + 2;                // warps 14, 15: V^T P^T issue for stream 0, 1
+constexpr int kLoadWarp0 = kPvWarp0 + 2;               // warps 16, 17: loader for stream 0, 1
+constexpr int NT = (kLoadWarp0 + 2) * 32;              // 576
 constexpr uint32_t kTmemCols = 512;
 // TMEM column map
 __host__ __device__ constexpr uint32_t col_s(int s, int buf) { return (uint32_t)(s * 2 + buf) * 64u; }
@@ -302,7 +304,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       for (int g = 0; g < 2; ++g) {
         tc::mbar_init(bar(s, B_SREADY + g), 1);
         tc::mbar_init(bar(s, B_SFREE + g), 2);
-        tc::mbar_init(bar(s, B_PREADY + g), 2);
+        tc::mbar_init(bar(s, B_PREADY + g), 6);  // 2 softmax warps (P written) + 4 correction warps (O rescaled)
         tc::mbar_init(bar(s, B_FREADY + g), 2);
         tc::mbar_init(bar(s, B_XREADY + g), 2);
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
@@ -385,7 +387,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     }
   }
   // =========================================================================================== MMA warps
-  else if (warp >= kMmaWarp0) {
+  else if (warp >= kMmaWarp0 && warp < kPvWarp0) {
     // The whole warp runs this loop with warp-uniform control flow and values; only the tcgen05 instructions
     // themselves are issued by one elected lane.  (Under a lane-0 branch every descriptor would have to be moved from
     // vector to uniform registers before each issue, which costs more than the MMA itself.)
@@ -400,16 +402,9 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       const uint64_t qd1 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][1]) - (s ? 1024u : 0u), 1024, 128);
       const uint64_t qd2 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][2]) - (s ? 1024u : 0u), 1024, 128);
       const uint64_t kd0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]), 1024, 128);
-      const uint64_t vd0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]), D * 16, 128);
       const uint64_t ksf0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]) + kSlots * D / 2, 128, 128);
-      const uint64_t vsf0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]) + D * kSlots / 2, 128, 128);
-      const uint64_t pd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.p[s][0]), 1024, 128),
-                              tc::smem_desc(tc::smem_u32(smem + sm.p[s][1]), 1024, 128)};
-      const uint64_t sfpd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][0]), 128, 128),
-                                tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][1]), 128, 128)};
-      const uint32_t kstep = sm.kstage >> 4, vstep = sm.vstage >> 4;
-      const uint32_t t_sfq = tmem + col_sfq(s), t_sfk = tmem + col_sfk(s), t_sfv = tmem + col_sfv(s),
-                     t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
+      const uint32_t kstep = sm.kstage >> 4;
+      const uint32_t t_sfq = tmem + col_sfq(s), t_sfk = tmem + col_sfk(s);
       if (S.n4 > 0) {  // Q scale factors go to TMEM once; the record carries them for rows 0..63 and again for rows
                        // 64..127, so the same atom serves either stream
         if (tc::elect_one()) {
@@ -419,71 +414,85 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
                                                          128, 128));
         }
       }
-      int kk = 0, vv = 0;
-      uint32_t kpar = 0, vpar = 0;
-      bool alive = true;
-      // S(j) = Q K(j)^T
-      auto issue_qk = [&](int j) {
+      int kk = 0;
+      uint32_t kpar = 0;
+      // the score tiles are double buffered, so Q K^T runs up to two steps ahead of the softmax
+      for (int j = 0; j < S.L; ++j) {
         const int g = j & 1;
-        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp))) { alive = false; return; }
-        if (!PROF_WAIT(1, wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp))) { alive = false; return; }
+        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp))) break;
+        if (!PROF_WAIT(1, wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp))) break;
         tc::fence_after_sync();
         PROF_T(mq0);
         const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
         const uint32_t d_s = tmem + col_s(s, g);
         if (tc::elect_one()) {
-        if (j >= S.n48) {
+          if (j >= S.n48) {
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
-        } else if (j >= S.n4) {
+            for (int ks = 0; ks < D / 16; ++ks) tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
+          } else if (j >= S.n4) {
 #pragma unroll
-          for (int ks = 0; ks < D / 32; ++ks) tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
-        } else {
-          const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
+            for (int ks = 0; ks < D / 32; ++ks) tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
+          } else {
+            const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
 #pragma unroll
-          for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
+            for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
 #pragma unroll
-          for (int ks = 0; ks < D / 64; ++ks)
-            tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks, t_sfk + 4 * ks);
-        }
-        tc::mma_commit(bar(s, B_SREADY + g));
-        tc::mma_commit(bar(s, B_KFREE + kk));
+            for (int ks = 0; ks < D / 64; ++ks)
+              tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks, t_sfk + 4 * ks);
+          }
+          tc::mma_commit(bar(s, B_SREADY + g));
+          tc::mma_commit(bar(s, B_KFREE + kk));
         }
         __syncwarp();
         PROF_T(mq1);
         PROF_ADD(5, mq0, mq1);
         if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
-      };
-      // the score tiles are double buffered, so Q K^T runs two steps ahead of the accumulation
-      issue_qk(0);
-      if (alive && S.L > 1) issue_qk(1);
-      for (int j = 0; j < S.L && alive; ++j) {
-        if (j + 2 < S.L) { issue_qk(j + 2); if (!alive) break; }
-        // ---- O^T += V(j)^T P(j)^T
+      }
+    }
+  }
+  // =========================================================================================== PV warps
+  else if (warp >= kPvWarp0) {
+    const int s = warp - kPvWarp0;
+    StreamInfo S = s ? st1 : st0;
+    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
+    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
+    S.L = __shfl_sync(0xffffffffu, S.L, 0);
+    if (S.L > 0) {
+      const uint64_t vd0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]), D * 16, 128);
+      const uint64_t vsf0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]) + D * kSlots / 2, 128, 128);
+      const uint64_t pd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.p[s][0]), 1024, 128),
+                              tc::smem_desc(tc::smem_u32(smem + sm.p[s][1]), 1024, 128)};
+      const uint64_t sfpd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][0]), 128, 128),
+                                tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][1]), 128, 128)};
+      const uint32_t vstep = sm.vstage >> 4;
+      const uint32_t t_sfv = tmem + col_sfv(s), t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
+      int vv = 0;
+      uint32_t vpar = 0;
+      for (int j = 0; j < S.L; ++j) {
+        // ---- O^T += V(j)^T P(j)^T, once P(j) is written and the accumulator is rescaled for step j
         const int g = j & 1;
         if (!PROF_WAIT(2, wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp))) break;
         if (!PROF_WAIT(3, wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp))) break;
-        if (!PROF_WAIT(4, wait_or_abort(bar(s, B_OCORR + g), (j >> 1) & 1, abortp))) break;
         tc::fence_after_sync();
         PROF_T(mp0);
         const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
         const uint32_t acc = j > 0;
         if (tc::elect_one()) {
-        if (j >= S.n48) {
+          if (j >= S.n48) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
-        } else if (j >= S.n4) {
+            for (int ks = 0; ks < 4; ++ks)
+              tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
+          } else if (j >= S.n4) {
 #pragma unroll
-          for (int ks = 0; ks < 2; ++ks)
-            tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
-        } else {
-          tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
-          tc::tmem_cp_sf(t_sfp, sfpd[g]);
-          tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
-        }
-        tc::mma_commit(bar(s, B_PVDONE + g));
-        tc::mma_commit(bar(s, B_VFREE + vv));
+            for (int ks = 0; ks < 2; ++ks)
+              tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
+          } else {
+            tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
+            tc::tmem_cp_sf(t_sfp, sfpd[g]);
+            tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
+          }
+          tc::mma_commit(bar(s, B_PVDONE + g));
+          tc::mma_commit(bar(s, B_VFREE + vv));
         }
         __syncwarp();
         PROF_T(mp1);
@@ -718,7 +727,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             tc::fence_before_sync();
           }
         }
-        warp_arrive(bar(s, B_OCORR + g));
+        warp_arrive(bar(s, B_PREADY + g));
       }
     }
     // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
@@ -769,7 +778,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 
 #ifdef DA2_PROF
   if (blockIdx.x == gridDim.x / 2 && lane == 0) {
-    const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == 8 ? 2 : warp == 12 ? 3 : warp == 14 ? 4 : -1;
+    const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == 8 ? 2 : warp == 12 ? 3 : warp == 16 ? 4 : warp == 14 ? 5 : -1;
     if (role >= 0) {
       prof_acc[7] = clock64() - prof_t0;
       for (int k = 0; k < 8; ++k) p.status[8 + role * 8 + k] = (int)(prof_acc[k] >> 4);  // units of 16 cycles
