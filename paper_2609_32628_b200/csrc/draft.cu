@@ -2,9 +2,11 @@
 //   logits[0][bh][a][b] = scale * Qavg_a . Kavg_b      logits[1][bh][a][b] = scale * Qmax_a . Kmax_b
 // The row softmaxes, their mixture and the ranking follow in rank.cu.
 //
-// The ranking compares scores to about 1e-5 relative, so the contraction is carried in fp32 FMAs (descriptor
-// values are fp32 means; rounding them to a 16-bit tensor-core format would reorder near-ties).  It is a small
-// GEMM: 4*R*R*d flops per head, against 4*64*64*d flops per retained block pair in the attention kernel.
+// The ranking compares scores to about 1e-5 relative and a softmax turns an ABSOLUTE logit error into a RELATIVE
+// score error, so the contraction accumulates in fp64 (products of fp32 descriptors are exact there) and only the
+// final logit is rounded to fp32; with large logits (outlier channels) fp32 accumulation alone would already move
+// scores by 1e-4.  It is a small GEMM: 4*R*R*d flops per head, against 4*64*64*d flops per retained block pair in
+// the attention kernel, so the fp64 rate is not a concern.
 // 64 x 64 output tile per CTA, 4 x 4 register tile per thread, K panel of 16 channels in shared memory.
 #include "da2_internal.cuh"
 
@@ -24,11 +26,11 @@ __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
   __shared__ float Bs[TK][TN + 4];
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;  // thread tile: rows ty*4.., cols tx*4..
-  float acc[4][4];
+  double acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
 
   // loader mapping: 64 rows x 16 channels = 256 float4 quarters -> one float4 per thread per matrix
   const int lr = tid >> 2, lc = (tid & 3) * 4;
@@ -44,11 +46,11 @@ __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
     for (int kk = 0; kk < TK; ++kk) {
       const float4 av = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
       const float4 bv = *reinterpret_cast<const float4 *>(&Bs[kk][tx * 4]);
-      const float ar[4] = {av.x, av.y, av.z, av.w}, br[4] = {bv.x, bv.y, bv.z, bv.w};
+      const double ar[4] = {av.x, av.y, av.z, av.w}, br[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma(ar[i], br[j], acc[i][j]);
     }
   }
 #pragma unroll
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int b = b0 + tx * 4 + j;
-      if (b < p.R) out[(size_t)a * p.R + b] = p.scale * acc[i][j];
+      if (b < p.R) out[(size_t)a * p.R + b] = (float)((double)p.scale * acc[i][j]);
     }
   }
 }

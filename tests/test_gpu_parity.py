@@ -213,3 +213,23 @@ def _sampled_parity(name, nheads=2, nblocks=6):
 
 def test_wan1p3b_480p_sampled_parity():
     _sampled_parity("wan1p3b_480p", nheads=2, nblocks=6)
+
+
+def test_hunyuan_720p_sampled_parity():
+    _sampled_parity("hunyuan_720p", nheads=1, nblocks=4)
+
+
+def test_wan14b_720p_sampled_parity():
+    """The benchmark's workload (20 % 8-bit + 40 % 4-bit, K outlier channels) in the benchmark's launch configuration."""
+    _sampled_parity("wan14b_720p", nheads=1, nblocks=4)
+
+
+def test_wan14b_720p_bf16_8bit_variant_sampled_parity():
+    _sampled_parity("wan14b_720p_hi", nheads=1, nblocks=4)
+
+
+def test_sweep_point_sampled_parity():
+    """One point of the budget sweep: 16 x 48 x 48 grid, 24 heads, 10 % 8-bit + 40 % 4-bit."""
+    w = da2_inputs.sweep_workload(2, 0.10, 0.40)
+    da2_inputs.WORKLOADS[w.name] = w
+    _sampled_parity(w.name, nheads=1, nblocks=4)
