@@ -104,14 +104,27 @@ def flop_counts(w, plan, ws):
     return dense, padded, valid
 
 
+def rank_workload(name: str, rank: int):
+    """Weak scaling: every rank runs the whole named workload on its own batch element (heads and batch elements never
+    mix on this path, so there is no collective); only the input seed differs per rank."""
+    base = da2_inputs.WORKLOADS[name]
+    return da2_inputs.Workload(**{**base.__dict__, "seed": base.seed + 1000 * rank})
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Step time of the job = the slowest rank's."""
+    if world <= 1:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_da2(args, rank, world, local_rank):
     import paper_2609_32628_b200 as da2
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
-    base = da2_inputs.WORKLOADS[args.workload]
-    # weak scaling: every rank runs the whole named workload on its own batch element (heads never mix, so there
-    # is no collective on the path); seeds differ per rank
-    w = da2_inputs.Workload(**{**base.__dict__, "seed": base.seed + 1000 * rank})
+    w = rank_workload(args.workload, rank)
     q, k, v = da2_inputs.make_qkv(w, dev)
     plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
                         rank_scope=args.rank_scope)
@@ -158,11 +171,7 @@ def run_da2(args, rank, world, local_rank):
     prep_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
     attn_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
     assert da2.da2_device_status(plan, ws) == 0, "device status after the timed region"
-    ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(total_ms / args.steps, world, dev)
 
     # ---- end to end through the C ABI with host buffers
     hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
@@ -187,11 +196,7 @@ def run_da2(args, rank, world, local_rank):
         e2e_step()
     a1.record(stream)
     barrier()
-    e2e_ms = a0.elapsed_time(a1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(a0.elapsed_time(a1) / e2e_steps, world, dev)
     if rank != 0:
         return None
 
