@@ -206,11 +206,11 @@ def run_da2(args, rank, world, local_rank):
     t_roof_nominal_ms = sum(padded[t] / (2.25e15 * NOMINAL_RATIO[t]) for t in range(3)) * 1e3
     total_valid = sum(valid)
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "attention_traffic.json")
+    tpath = os.path.join(ROOT, "profiles", "attention_kernel_dram_traffic.txt")
     if os.path.exists(tpath):
-        tj = json.load(open(tpath))
-        if tj.get("workload") == args.workload:
-            traffic = tj.get("dram_bytes_per_launch")
+        for ln in open(tpath):
+            if ln.startswith("workload=" + args.workload + " "):
+                traffic = int(ln.split("dram_bytes_per_launch=")[1].split()[0])
     roofline = {
         "kernel": "attention_kernel (da2_attention_fwd)", "bound": "tensor",
         "achieved": total_valid / (attn_ms * 1e-3) / 1e12,
