@@ -136,6 +136,23 @@ def sweep_workload(grid_index: int, high: float, low: float, *, high_is_bf16: bo
                     seed=100 + grid_index)
 
 
+def _register_sweep():
+    """Budget sweep at the largest and smallest grids plus the dense endpoints, as named workloads."""
+    names = {0: "8k", 1: "16k", 2: "37k", 3: "65k", 4: "131k"}
+    for gi in (0, 2, 4):
+        for high, low in ((0.05, 0.20), (0.10, 0.40), (0.20, 0.60)):
+            w = sweep_workload(gi, high, low)
+            WORKLOADS[f"sweep_{names[gi]}_{int(high * 100)}_{int(low * 100)}"] = Workload(
+                **{**w.__dict__, "name": f"sweep_{names[gi]}_{int(high * 100)}_{int(low * 100)}"})
+    w = sweep_workload(4, 1.0, 0.0)
+    WORKLOADS["sweep_131k_all8"] = Workload(**{**w.__dict__, "name": "sweep_131k_all8"})
+    w = sweep_workload(4, 1.0, 0.0, high_is_bf16=True)
+    WORKLOADS["sweep_131k_allbf16"] = Workload(**{**w.__dict__, "name": "sweep_131k_allbf16"})
+
+
+_register_sweep()
+
+
 def make_tensor(w: Workload, tensor_id: int, device="cpu", heads=None) -> torch.Tensor:
     """bf16 [B, H', N, d] tensor number `tensor_id` (0=Q, 1=K, 2=V) of workload `w`.
 
