@@ -40,11 +40,11 @@ namespace da2 {
 
 namespace {
 
-constexpr int kSoftmaxWarps = 16, kCorrWarps = 4;
-constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // Q K^T issue for stream 0, 1
-constexpr int kPvWarp0 = kMmaWarp0 + 2;                // V^T P^T issue for stream 0, 1
-constexpr int kLoadWarp0 = kPvWarp0 + 2;               // loader for stream 0, 1
-constexpr int NT = (kLoadWarp0 + 2) * 32;              // 832
+constexpr int kSoftmaxWarps = 8, kCorrWarps = 4;
+constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // warps 12, 13: Q K^T issue for stream 0, 1
+constexpr int kPvWarp0 = kMmaWarp0 + 2;                // warps 14, 15: V^T P^T issue for stream 0, 1
+constexpr int kLoadWarp0 = kPvWarp0 + 2;               // warps 16, 17: loader for stream 0, 1
+constexpr int NT = (kLoadWarp0 + 2) * 32;              // 576
 constexpr uint32_t kTmemCols = 512;
 // TMEM column map
 __host__ __device__ constexpr uint32_t col_s(int s, int buf) { return (uint32_t)(s * 2 + buf) * 64u; }
@@ -62,8 +62,8 @@ constexpr float kOffsetP8 = 8.807f;      // base-2 exponent offset (about log2 4
 // barrier indices inside one stream's group
 // (a parity wait can only tell the latest completion from the one before, so every barrier is laid out such that no
 // waiter can fall two completions behind: buffers indexed by step parity get one barrier per buffer)
-enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_HX = 22,
-       B_XREADY = 24, B_PVDONE = 26, B_HX2 = 28, B_ELL = 30, B_Q = 31, B_COUNT = 32 };
+enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_FREADY = 22,
+       B_XREADY = 24, B_PVDONE = 26, B_OCORR = 28, B_ELL = 30, B_Q = 31, B_COUNT = 32 };
 constexpr int kMaxStages = 4, kInfoRing = 8;
 
 struct SmemMap {
@@ -76,8 +76,8 @@ struct SmemMap {
   uint32_t sfp[2][2]; // P scale atoms (512 B)
   uint32_t factor;    // float [2 streams][2][64]
   uint32_t changed;   // uint8 [2][2][64]
-  uint32_t xmax;      // float [2 streams][4 step slots + 2 final references][64]
-  uint32_t ell;       // float [2 streams][2 sets][2 column halves][64]
+  uint32_t xmax;      // float [2][2 parity][2 halves][64]
+  uint32_t ell;       // float [2][2 halves][64]
   uint32_t info;      // per stream, ring of kInfoRing steps: {u64 mask, float dk8, pad}
   uint32_t bars;      // uint64 [2][B_COUNT]
   uint32_t kstage, vstage;  // bytes per ring stage
@@ -103,7 +103,7 @@ __host__ SmemMap make_smem_map(const Params &p) {
   const uint32_t q_end = cur;
   const uint32_t pbytes = p.tier_active[2] ? 8192u : (p.tier_active[1] ? 4096u : 2048u);
   // ring depths: as deep as shared memory allows (the K ring also serves as the 16 KB output staging tile)
-  const uint32_t fixed = 4 * pbytes + (pbytes > 2048u ? 0 : 4 * 512) + 1024 + 256 + 3072 + 2048 + 2 * kInfoRing * 16 +
+  const uint32_t fixed = 4 * pbytes + 4 * 512 + 1024 + 256 + 2048 + 1024 + 2 * kInfoRing * 16 +
                          2 * B_COUNT * 8 + 1024;
   const uint32_t budget = 232448u - q_end - fixed;
   const int cand[5][2] = {{4, 4}, {3, 4}, {3, 3}, {2, 3}, {2, 2}};
@@ -119,14 +119,12 @@ __host__ SmemMap make_smem_map(const Params &p) {
   for (int s = 0; s < 2; ++s)
     for (int g = 0; g < kMaxStages; ++g) m.vst[s][g] = g < m.nv ? take(vstage) : 0;
   for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.p[s][g] = take(pbytes);
-  // the NVFP4 weights fill 2 KB of a P buffer; where the buffer is larger (another tier is active) their scale atom
-  // lives in its upper part
-  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.sfp[s][g] = pbytes > 2048u ? m.p[s][g] + 2048u : take(512);
+  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.sfp[s][g] = take(512);
   m.factor = take(2 * 2 * 64 * 4);
   m.changed = take(2 * 2 * 64);
   m.chg = take(2 * 2 * 2 * 4);
-  m.xmax = take(2 * 6 * 64 * 4);
-  m.ell = take(2 * 2 * 2 * 64 * 4);
+  m.xmax = take(2 * 2 * 2 * 64 * 4);
+  m.ell = take(2 * 2 * 64 * 4);
   m.info = take(2 * kInfoRing * 16);
   m.bars = take(2 * B_COUNT * 8);
   m.total = cur;
@@ -290,8 +288,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   auto bar = [&](int s, int which) -> uint64_t * { return bars + s * B_COUNT + which; };
   float *s_factor = reinterpret_cast<float *>(smem + sm.factor);      // [s][buf][64]
   uint32_t *s_chg = reinterpret_cast<uint32_t *>(smem + sm.chg);      // [s][buf][2]
-  float *s_xmax = reinterpret_cast<float *>(smem + sm.xmax);          // [s][4 slots + 2 references][64]
-  float *s_ell = reinterpret_cast<float *>(smem + sm.ell);            // [s][set][column half][64]
+  float *s_xmax = reinterpret_cast<float *>(smem + sm.xmax);          // [s][parity][half][64]
+  float *s_ell = reinterpret_cast<float *>(smem + sm.ell);            // [s][half][64]
   uint8_t *s_info = smem + sm.info;                                   // [s][kInfoRing] 16 bytes
 
   if (warp == 0) {
@@ -302,12 +300,12 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     for (int s = 0; s < 2; ++s) {
       for (int g = 0; g < 2; ++g) {
         tc::mbar_init(bar(s, B_SREADY + g), 1);
-        tc::mbar_init(bar(s, B_SFREE + g), 4);
-        tc::mbar_init(bar(s, B_PREADY + g), 8);  // 4 softmax warps (P written) + 4 correction warps (O rescaled)
-        tc::mbar_init(bar(s, B_HX + g), 2);   // rows 0..31: the two column halves of set g
-        tc::mbar_init(bar(s, B_HX2 + g), 2);  // rows 32..63
+        tc::mbar_init(bar(s, B_SFREE + g), 2);
+        tc::mbar_init(bar(s, B_PREADY + g), 6);  // 2 softmax warps (P written) + 4 correction warps (O rescaled)
+        tc::mbar_init(bar(s, B_FREADY + g), 2);
         tc::mbar_init(bar(s, B_XREADY + g), 2);
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
+        tc::mbar_init(bar(s, B_OCORR + g), 4);
       }
       for (int g = 0; g < kMaxStages; ++g) {
         tc::mbar_init(bar(s, B_FULLK + g), 1);
@@ -315,7 +313,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         tc::mbar_init(bar(s, B_KFREE + g), 1);
         tc::mbar_init(bar(s, B_VFREE + g), 1);
       }
-      tc::mbar_init(bar(s, B_ELL), 8);
+      tc::mbar_init(bar(s, B_ELL), 4);
       tc::mbar_init(bar(s, B_Q), 1);
     }
     tc::fence_barrier_init();
@@ -537,24 +535,21 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   }
   // =========================================================================================== softmax warps
   else if (warp < kSoftmaxWarps) {
-    // Sixteen warps: TMEM lane quarter q = warp & 3 (stream q >> 1, rows 32 * (q & 1) ..), step parity ("set")
-    // (warp >> 2) & 1, column half warp >> 3.  A thread owns 32 of the 64 keys of one query row in every other step.
-    // The four warps of a scheduler thus hold two steps in flight, each split in two: while some exponentiate and
-    // pack (special-function bound), the others fetch, mask and reduce.  Hand-offs: the block maxima of the two halves
-    // of a row (between the two warps of a step), and the running maximum (from one step to the next).
-    const int q4 = warp & 3, s = q4 >> 1, rh = q4 & 1, par = (warp >> 2) & 1, ch = warp >> 3;
-    const int r = rh * 32 + lane;  // query row inside the stream's block
+    // The two softmax warps that share a scheduler (warp w and w+4) own the same 32 query rows and take ALTERNATE
+    // steps, one thread per full 64-key row: while one exponentiates and packs its step (special-function bound),
+    // the other fetches, masks and reduces the next one.  The only hand-off between them is the running maximum.
+    const int s = (warp & 3) >> 1, par = warp >> 2;
+    const int r = (warp & 1) * 32 + lane;  // query row inside the stream's block
     const StreamInfo S = s ? st1 : st0;
-    const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const float gqk = p.gscale[bh * 4 + 0] * p.gscale[bh * 4 + 1] * p.scale * kLog2e;
     const float dq8s = (S.a >= 0 && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
     const float c16 = p.scale * kLog2e;
     float h_own = -INFINITY, ell = 0.f;  // log2-domain maximum after this warp's last step; its partial denominator
     const int g = par;                   // buffers of this warp's step parity
-    // running maximum after step i: slot i & 3 (step i+4 may overwrite it only after every reader of step i+1 is past)
-    float *h_ring = s_xmax + s * 6 * 64 + r;
-    uint64_t *hx = bar(s, (rh ? B_HX2 : B_HX) + g);
-    const uint32_t s_col = tmem + lane_addr + col_s(s, g) + ch * 32;
+    float *my_h = s_xmax + ((s * 2 + g) * 2 + 0) * 64 + r;           // published running maximum of my steps
+    const float *other_h = s_xmax + ((s * 2 + (g ^ 1)) * 2 + 0) * 64 + r;
+    const uint32_t s_col = tmem + lane_addr + col_s(s, g);
     uint8_t *prow = smem + sm.p[s][g] + r * 16;
 
     for (int i = par; i < S.L; i += 2) {
@@ -563,11 +558,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       if (!PROF_WAIT(0, wait_or_abort(bar(s, B_SREADY + g), kp, abortp))) break;
       tc::fence_after_sync();
       PROF_T(pt0);
-      float v[32];
+      float v[64];
       {
-        uint32_t a0[16], a1[16];
+        uint32_t a0[16], a1[16], a2[16], a3[16];
         tc::tmem_ld16(s_col, a0);
         tc::tmem_ld16(s_col + 16, a1);
+        tc::tmem_ld16(s_col + 32, a2);
+        tc::tmem_ld16(s_col + 48, a3);
         tc::wait_ld();
         // int32 accumulators become floats exactly through a magic-number add and subtract (|S| < 2^22): two
         // full-rate operations instead of a conversion on the special-function unit
@@ -577,11 +574,14 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           for (int c = 0; c < 16; c += 2) {
             unf2(add2(f2(__uint_as_float(a0[c] + 0x4B400000u), __uint_as_float(a0[c + 1] + 0x4B400000u)), moff), v[c], v[c + 1]);
             unf2(add2(f2(__uint_as_float(a1[c] + 0x4B400000u), __uint_as_float(a1[c + 1] + 0x4B400000u)), moff), v[16 + c], v[17 + c]);
+            unf2(add2(f2(__uint_as_float(a2[c] + 0x4B400000u), __uint_as_float(a2[c + 1] + 0x4B400000u)), moff), v[32 + c], v[33 + c]);
+            unf2(add2(f2(__uint_as_float(a3[c] + 0x4B400000u), __uint_as_float(a3[c + 1] + 0x4B400000u)), moff), v[48 + c], v[49 + c]);
           }
         } else {
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
             v[c] = __uint_as_float(a0[c]); v[16 + c] = __uint_as_float(a1[c]);
+            v[32 + c] = __uint_as_float(a2[c]); v[48 + c] = __uint_as_float(a3[c]);
           }
         }
       }
@@ -590,45 +590,39 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       tc::fence_before_sync();
       warp_arrive(bar(s, B_SFREE + g));
       const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
-      const uint32_t kmask = *reinterpret_cast<const uint32_t *>(info + 4 * ch);
+      const uint2 kmask = *reinterpret_cast<const uint2 *>(info);
       float coef;
       if (tier == 2) coef = c16;
       else if (tier == 1) coef = dq8s * *reinterpret_cast<const float *>(info + 8);
       else coef = gqk;
-      if (kmask != 0xffffffffu) {  // ragged edge tile: padding keys take no part
+      if ((kmask.x & kmask.y) != 0xffffffffu) {  // ragged edge tile: padding keys take no part
 #pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = ((kmask >> c) & 1u) ? v[c] : -INFINITY;
+        for (int c = 0; c < 32; ++c) {
+          v[c] = ((kmask.x >> c) & 1u) ? v[c] : -INFINITY;
+          v[32 + c] = ((kmask.y >> c) & 1u) ? v[32 + c] : -INFINITY;
+        }
       }
-      // maxima of the two 16-key groups, then of this half of the row; the other half's comes through shared memory
-      float gm[2];
-      gm[0] = max16(v);
-      gm[1] = max16(v + 16);
-      const float hmax = fmaxf(gm[0], gm[1]) * coef;  // log2 domain
+      // maxima of the four 16-key groups (pairwise trees), then of the row
+      float gm[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) gm[q] = max16(v + q * 16);
+      const float pmax = fmaxf(max3(gm[0], gm[1], gm[2]), gm[3]) * coef;  // log2 domain
       PROF_T(pt2);
       PROF_ADD(4, pt1, pt2);
       // PV(i-2) done: this parity's P buffer is free and the correction warps are past step i-2
       if (i >= 2 && !PROF_WAIT(1, wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp))) break;
-      // The two halves of a row exchange their block maxima through the free P buffer: each writes into the first
-      // 16-byte chunk of the OTHER half's part of the row, which only that half overwrites later (with its weights).
-      const int cph = tier == 2 ? 4 : (tier == 1 ? 2 : 1);  // 16-byte chunks per column half
-      *reinterpret_cast<float *>(prow + (ch ^ 1) * cph * 1024) = hmax;
-      warp_arrive(hx);
-      if (!PROF_WAIT(1, wait_or_abort(hx, kp, abortp))) break;
-      const float pmax = fmaxf(hmax, *reinterpret_cast<const float *>(prow + ch * cph * 1024));
-      // running maximum after step i-1, published by the previous step's warps
+      // running maximum after step i-1, published by the other warp
       float h_prev = -INFINITY;
       if (i > 0) {
         if (!PROF_WAIT(2, wait_or_abort(bar(s, B_XREADY + (g ^ 1)), (uint32_t)((i - 1) >> 1) & 1u, abortp))) break;
-        h_prev = h_ring[((i - 1) & 3) * 64];
+        h_prev = *other_h;
       }
       const float m_new = fmaxf(h_prev, pmax);
-      if (ch == 0) {  // both halves hold the same values; one publishes them
-        h_ring[(i & 3) * 64] = m_new;
-        s_factor[(s * 2 + g) * 64 + r] = ex2(h_prev - m_new);  // 0 on the first block (h_prev = -inf)
-        const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h_prev);
-        if (lane == 0) s_chg[(s * 2 + g) * 2 + rh] = moved;
-        warp_arrive(bar(s, B_XREADY + g));  // the next step's warps and the correction warps wait on this
-      }
+      *my_h = m_new;
+      s_factor[(s * 2 + g) * 64 + r] = ex2(h_prev - m_new);  // 0 on the first block (h_prev = -inf)
+      const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h_prev);
+      if (lane == 0) s_chg[(s * 2 + g) * 2 + (warp & 1)] = moved;
+      warp_arrive(bar(s, B_XREADY + g));  // the other warp's next step and the correction warps wait on this
       ell *= ex2(h_own - m_new);
       h_own = m_new;
 
@@ -638,7 +632,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         const uint64_t bias2 = f2(-m_new, -m_new);
         uint64_t sum2 = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 8; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -647,7 +641,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             sum2 = add2(sum2, f2(w0, w1));
             w4[j] = pack_bf16x2(w0, w1);
           }
-          *reinterpret_cast<uint4 *>(prow + (ch * 4 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         float s0, s1;
         unf2(sum2, s0, s1);
@@ -656,7 +650,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         const uint64_t bias2 = f2(kOffsetP8 - m_new, kOffsetP8 - m_new);
         uint64_t sum2 = 0;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < 4; ++c) {
           uint32_t w4[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -666,21 +660,20 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             sum2 = add2(add2(sum2, f2(w0, w1)), f2(w2, w3));
             w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
           }
-          *reinterpret_cast<uint4 *>(prow + (ch * 2 + c) * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         float s0, s1;
         unf2(sum2, s0, s1);
         ell += kEtaP8 * (s0 + s1);  // the denominator sums the amplified fp32 weights; eta restores the unit
       } else {
-        uint32_t sfhalf = 0;
-        uint32_t cw[4];
+        uint32_t sfword = 0;
 #pragma unroll
-        for (int gi = 0; gi < 2; ++gi) {
+        for (int gi = 0; gi < 4; ++gi) {
           // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent:
           // sigma = E4M3(448 * max w); scaled weight u = w * 2688 / sigma = 2^(x - m + log2(2688) - log2(sigma))
           const float gw = ex2(fmaf(gm[gi], coef, -m_new));
           const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gw), 0.f) & 0xffu;
-          sfhalf |= sc << (8 * gi);
+          sfword |= sc << (8 * gi);
           // E4M3 code -> fp32: for normal codes the bit pattern is a shift and a re-bias; the 7 subnormal codes
           // and zero (weights below 2^-15 of the row maximum) take the general conversion
           const float sigma = sc >= 8u ? __uint_as_float((sc << 20) + 0x3C000000u) : decode_e4m3(sc);
@@ -698,15 +691,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             const uint32_t pk = pack_e2m1x4(u0, u1, u2, u3);
             if (j < 2) c0 |= pk << (16 * j); else c1 |= pk << (16 * (j - 2));
           }
-          cw[gi * 2 + 0] = live ? c0 : 0u;
-          cw[gi * 2 + 1] = live ? c1 : 0u;
+          // 16 keys = 8 bytes: chunk gi/2 (32 keys per 16-byte chunk), half gi&1
+          *reinterpret_cast<uint2 *>(prow + (gi >> 1) * 1024 + (gi & 1) * 8) = make_uint2(live ? c0 : 0u, live ? c1 : 0u);
           float s0, s1;
           unf2(sum2, s0, s1);
           ell = fmaf(s0 + s1, live ? sigma * (1.0f / 2688.0f) : 1.0f, ell);
         }
-        // 32 keys = one 16-byte chunk of the row (chunk index = column half)
-        *reinterpret_cast<uint4 *>(prow + ch * 1024) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-        *reinterpret_cast<uint16_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4 + ch * 2) = (uint16_t)sfhalf;
+        *reinterpret_cast<uint32_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4) = sfword;
       }
       PROF_T(pt4);
       PROF_ADD(5, pt3, pt4);
@@ -716,8 +707,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       PROF_ADD(6, pt4, pt5);
     }
     if (S.L > 0) {
-      s_ell[((s * 2 + par) * 2 + ch) * 64 + r] = ell;
-      if (ch == 0) s_xmax[(s * 6 + 4 + par) * 64 + r] = h_own;  // reference of this set's partial denominators
+      s_ell[(s * 2 + par) * 64 + r] = ell;
+      s_xmax[((s * 2 + par) * 2 + 1) * 64 + r] = h_own;  // reference of this partial denominator
       warp_arrive(bar(s, B_ELL));
     }
   }
@@ -793,11 +784,10 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const int qr = c * 8 + j;
-              // the four warps of a row kept partial denominators relative to their set's last maximum
-              const float h0 = s_xmax[(s * 6 + 4) * 64 + qr], h1 = s_xmax[(s * 6 + 5) * 64 + qr];
+              // the two warps of a row kept partial denominators relative to their own last maximum
+              const float h0 = s_xmax[((s * 2 + 0) * 2 + 1) * 64 + qr], h1 = s_xmax[((s * 2 + 1) * 2 + 1) * 64 + qr];
               const float hf = fmaxf(h0, h1);
-              const float l = (s_ell[((s * 2 + 0) * 2 + 0) * 64 + qr] + s_ell[((s * 2 + 0) * 2 + 1) * 64 + qr]) * ex2(h0 - hf) +
-                              (s_ell[((s * 2 + 1) * 2 + 0) * 64 + qr] + s_ell[((s * 2 + 1) * 2 + 1) * 64 + qr]) * ex2(h1 - hf);
+              const float l = s_ell[(s * 2 + 0) * 64 + qr] * ex2(h0 - hf) + s_ell[(s * 2 + 1) * 64 + qr] * ex2(h1 - hf);
               const float val = l > 0.f ? __uint_as_float(o[j]) * unit * __fdiv_rn(1.0f, l) : 0.f;
               stage[qr * D + ch] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
             }
