@@ -115,6 +115,17 @@ da2_status_t da2_plan_info(const da2_plan_t *plan, da2_plan_info_t *info);
 da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
                          size_t workspace_bytes, void *stream);
 
+/* Operands only.  The paper reuses the token-to-region partition across layers and denoising steps (Sec. 3.3,
+ * "Fused quantization and reordering"): that is the plan object, which any number of calls may share.  This entry
+ * point goes one step further on the caller's responsibility (the paper has no counterpart): it recomputes the
+ * statistics, scales and operand records of (q, k, v) in a workspace that an earlier da2_prepare with the same plan
+ * filled, and leaves that call's draft map, counts and id lists untouched, so that the selection of one call can
+ * serve a later one.  Same argument rules as da2_prepare; the region descriptors are refreshed as a by-product.  In a
+ * workspace that no da2_prepare has filled there are no lists: da2_attention_fwd then reads undefined ids (an id
+ * out of range is reported through the status word, its row's output is undefined).  Enqueues on stream. */
+da2_status_t da2_refresh_operands(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+
 /* Phased mixed-precision block-sparse attention.  workspace must have been filled by da2_prepare for the same
  * q, k, v (ordering on the same stream is enough).  Rows whose list is empty give zeros (App. C.1). */
 da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,

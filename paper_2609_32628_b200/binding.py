@@ -62,6 +62,8 @@ def load_library():
         lib.da2_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
         lib.da2_prepare.restype = ctypes.c_int
         lib.da2_prepare.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+        lib.da2_refresh_operands.restype = ctypes.c_int
+        lib.da2_refresh_operands.argtypes = [vp, vp, vp, vp, vp, sz, vp]
         lib.da2_attention_fwd.restype = ctypes.c_int
         lib.da2_attention_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         lib.da2_device_status.restype = ctypes.c_int
@@ -142,6 +144,14 @@ def da2_prepare(plan: Plan, q, k, v, workspace, stream=None) -> None:
                                     workspace.numel() * workspace.element_size(), _stream(stream))
     if rc != 0:
         raise Da2Error(rc, "da2_prepare")
+
+
+def da2_refresh_operands(plan: Plan, q, k, v, workspace, stream=None) -> None:
+    """q, k, v: CUDA bf16 [B,H,N,d] contiguous; workspace: CUDA uint8 tensor of plan.info.workspace_bytes."""
+    rc = load_library().da2_refresh_operands(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_refresh_operands")
 
 
 def da2_attention_fwd(plan: Plan, q, k, v, workspace, out, stream=None) -> None:

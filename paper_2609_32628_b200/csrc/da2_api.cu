@@ -175,8 +175,11 @@ da2_status_t da2_plan_info(const da2_plan_t *plan, da2_plan_info_t *info) {
   return DA2_OK;
 }
 
-da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
-                         size_t workspace_bytes, void *stream) {
+namespace {
+
+// da2_prepare and da2_refresh_operands: the same pipeline with or without the selection stages
+da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
+                          size_t workspace_bytes, void *stream, bool select) {
   if (!plan || !q || !k || !v || !workspace) return DA2_ERR_INVALID_ARG;
   if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(workspace, 256))
     return DA2_ERR_INVALID_ARG;
@@ -197,11 +200,25 @@ da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, c
                           (size_t)p.BH, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return DA2_ERR_CUDA;
   }
-  if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
-  if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  if (select) {
+    if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  }
   if (da2::launch_prep(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   plan->last_launches = launches;
   return DA2_OK;
+}
+
+}  // namespace
+
+da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,
+                         size_t workspace_bytes, void *stream) {
+  return prepare_impl(plan, q, k, v, workspace, workspace_bytes, stream, true);
+}
+
+da2_status_t da2_refresh_operands(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                                  void *workspace, size_t workspace_bytes, void *stream) {
+  return prepare_impl(plan, q, k, v, workspace, workspace_bytes, stream, false);
 }
 
 da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,

@@ -30,6 +30,8 @@ SMALL = {
     "all4": W("all4", 1, 1, 128, 2, 16, 16, 0.0, 0.0, 1.0, seed=15),
     # a 4 -> 16 switch with no 8-bit phase
     "skip8": W("skip8", 1, 2, 64, 2, 16, 16, 0.25, 0.0, 0.5, seed=16),
+    # batch of two (heads of different batch entries are independent problems), all three tiers
+    "batch2": W("batch2", 2, 2, 64, 2, 16, 16, 0.1, 0.2, 0.3, seed=17),
 }
 
 
@@ -233,3 +235,33 @@ def test_sweep_point_sampled_parity():
     w = da2_inputs.sweep_workload(2, 0.10, 0.40)
     da2_inputs.WORKLOADS[w.name] = w
     _sampled_parity(w.name, nheads=1, nblocks=4)
+
+
+def test_refresh_operands_keeps_the_selection():
+    """da2_refresh_operands: new operands under the lists of an earlier call (the selection is reused)."""
+    w1 = SMALL["ragged64"]
+    w2 = W("ragged64b", w1.B, w1.H, w1.head_dim, w1.T, w1.Hg, w1.Wg, w1.frac16, w1.frac8, w1.frac4, seed=112)
+    q1, k1, v1 = _inputs(w1)
+    q2, k2, v2 = _inputs(w2)
+    plan, ws, _ = run_gpu(w1, q1, k1, v1, zero_ws=True)
+    ref1 = oracle_all(w1, q1, k1, v1)
+    bad = _check_prepare(w1, plan, ws, ref1)
+    I = plan.info
+    keep = [(I.off_map, I.off_counts - I.off_map), (I.off_counts, I.off_ids - I.off_counts),
+            (I.off_ids, I.B * I.H * I.ids_per_head * 2)]
+    before = [ws[o:o + n].clone() for o, n in keep]
+    out = torch.full_like(q2, float("nan"))
+    da2.da2_refresh_operands(plan, q2, k2, v2, ws)
+    da2.da2_attention_fwd(plan, q2, k2, v2, ws, out)
+    torch.cuda.synchronize()
+    assert da2.da2_device_status(plan, ws) == 0
+    for (o, n), b in zip(keep, before):
+        assert torch.equal(ws[o:o + n], b), "the draft map, counts and ids must not change"
+    # operands, scales and descriptors are those of the new inputs: the oracle's, bit for bit
+    ref2 = oracle_all(w2, q2, k2, v2)
+    mixed = dict(ref2)
+    mixed.update(A=ref1["A"], ids=ref1["ids"], counts=ref1["counts"], tags=ref1["tags"])
+    assert _check_prepare(w2, plan, ws, mixed) == bad
+    sel = [(h, a) for h in range(w1.B * w1.H) for a in range(I.R)]
+    _check_attention(w2, out, mixed, sel, bad)
+    assert torch.isfinite(out.float()).all()
