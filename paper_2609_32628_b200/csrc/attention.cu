@@ -62,8 +62,8 @@ constexpr float kOffsetP8 = 8.807f;      // base-2 exponent offset (about log2 4
 // barrier indices inside one stream's group
 // (a parity wait can only tell the latest completion from the one before, so every barrier is laid out such that no
 // waiter can fall two completions behind: buffers indexed by step parity get one barrier per buffer)
-enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_FREADY = 22,
-       B_XREADY = 24, B_PVDONE = 26, B_OCORR = 28, B_ELL = 30, B_Q = 31, B_COUNT = 32 };
+enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_XREADY = 22,
+       B_PVDONE = 24, B_ELL = 26, B_Q = 27, B_COUNT = 28 };
 constexpr int kMaxStages = 4, kInfoRing = 8;
 
 struct SmemMap {
@@ -75,7 +75,6 @@ struct SmemMap {
   uint32_t p[2][2];   // P operand images per stream, double buffered (64 x 64 x <= 2 bytes)
   uint32_t sfp[2][2]; // P scale atoms (512 B)
   uint32_t factor;    // float [2 streams][2][64]
-  uint32_t changed;   // uint8 [2][2][64]
   uint32_t xmax;      // float [2][2 parity][2 halves][64]
   uint32_t ell;       // float [2][2 halves][64]
   uint32_t info;      // per stream, ring of kInfoRing steps: {u64 mask, float dk8, pad}
@@ -121,7 +120,6 @@ __host__ SmemMap make_smem_map(const Params &p) {
   for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.p[s][g] = take(pbytes);
   for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.sfp[s][g] = take(512);
   m.factor = take(2 * 2 * 64 * 4);
-  m.changed = take(2 * 2 * 64);
   m.chg = take(2 * 2 * 2 * 4);
   m.xmax = take(2 * 2 * 2 * 64 * 4);
   m.ell = take(2 * 2 * 64 * 4);
@@ -302,10 +300,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         tc::mbar_init(bar(s, B_SREADY + g), 1);
         tc::mbar_init(bar(s, B_SFREE + g), 2);
         tc::mbar_init(bar(s, B_PREADY + g), 6);  // 2 softmax warps (P written) + 4 correction warps (O rescaled)
-        tc::mbar_init(bar(s, B_FREADY + g), 2);
         tc::mbar_init(bar(s, B_XREADY + g), 2);
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
-        tc::mbar_init(bar(s, B_OCORR + g), 4);
       }
       for (int g = 0; g < kMaxStages; ++g) {
         tc::mbar_init(bar(s, B_FULLK + g), 1);

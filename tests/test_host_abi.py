@@ -71,3 +71,5 @@ def test_compute_calls_reject_null_pointers_without_touching_cuda():
     assert lib.da2_prepare(plan.handle, None, None, None, None, 0, None) == 1
     assert lib.da2_attention_fwd(plan.handle, None, None, None, None, None, None) == 1
     assert lib.da2_prepare(plan.handle, 16, 16, 16, 256, 10, None) == 3   # workspace too small, still no launch
+    assert lib.da2_refresh_operands(plan.handle, None, None, None, None, 0, None) == 1
+    assert lib.da2_refresh_operands(plan.handle, 16, 16, 16, 256, 10, None) == 3
