@@ -201,18 +201,26 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
 
 // bounded wait that also gives up as soon as another thread of the CTA has flagged a failure
 // (the flag then holds 1 + the shared-memory offset of the barrier that was never completed, for diagnosis)
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-  if (tc::mbar_try_wait(bar, parity)) return true;
-  // Waiting warps share their scheduler with the warps doing the softmax arithmetic, so they must not spin: each
-  // try suspends in hardware until the phase completes (or 20 us pass).  The bound is on elapsed clock cycles.
+//
+// Waiting warps share their scheduler with the warps doing the softmax arithmetic.  A plain mbarrier.try_wait blocks
+// in hardware for a while before it reports failure, so the retry loop issues few instructions (the variant with an
+// explicit time hint is expanded into a polling loop with nanosleep and clock reads: more instructions, same run
+// time).  The bound is on elapsed clock cycles, checked once per 16 tries.
+__device__ __forceinline__ bool wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
   const long long t0 = clock64();
   for (;;) {
-    if (tc::mbar_try_wait_suspend(bar, parity, 20000u)) return true;
+#pragma unroll 1
+    for (int k = 0; k < 16; ++k)
+      if (tc::mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (clock64() - t0 > 400000000ll) break;  // about 0.2 s
   }
   atomicCAS(const_cast<int *>(abort_flag), 0, 1 + (int)(tc::smem_u32(bar) & 0xffff));
   return false;
+}
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+  if (tc::mbar_try_wait(bar, parity)) return true;
+  return wait_slow(bar, parity, abort_flag);
 }
 
 #ifdef DA2_PROF
