@@ -632,76 +632,88 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 
       PROF_T(pt3);
       const uint64_t coef2 = f2(coef, coef);
-      if (tier == 2) {
-        const uint64_t bias2 = f2(-m_new, -m_new);
+      if (tier != 0) {
+        // the scores of the row become the exponent arguments, then the weights, in place: all 64 exponentials are
+        // issued before any is consumed (the 8-bit path carries the 2^8.807 offset in the exponent)
+        const float b = tier == 1 ? kOffsetP8 - m_new : -m_new;
+        const uint64_t bias2 = f2(b, b);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) unf2(fma2(f2(v[2 * j], v[2 * j + 1]), coef2, bias2), v[2 * j], v[2 * j + 1]);
+#pragma unroll
+        for (int j = 0; j < 64; ++j) v[j] = ex2(v[j]);
         uint64_t sum2 = 0;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint32_t w4[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float w0, w1;
-            exp_pair(v[c * 8 + 2 * j], v[c * 8 + 2 * j + 1], coef2, bias2, w0, w1);
-            sum2 = add2(sum2, f2(w0, w1));
-            w4[j] = pack_bf16x2(w0, w1);
-          }
-          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-        }
+        for (int j = 0; j < 32; j += 2) sum2 = add2(sum2, add2(f2(v[2 * j], v[2 * j + 1]), f2(v[2 * j + 2], v[2 * j + 3])));
         float s0, s1;
         unf2(sum2, s0, s1);
-        ell += s0 + s1;
-      } else if (tier == 1) {
-        const uint64_t bias2 = f2(kOffsetP8 - m_new, kOffsetP8 - m_new);
-        uint64_t sum2 = 0;
+        if (tier == 2) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t w4[4];
+          for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4 *>(prow + c * 1024) =
+                make_uint4(pack_bf16x2(v[c * 8 + 0], v[c * 8 + 1]), pack_bf16x2(v[c * 8 + 2], v[c * 8 + 3]),
+                           pack_bf16x2(v[c * 8 + 4], v[c * 8 + 5]), pack_bf16x2(v[c * 8 + 6], v[c * 8 + 7]));
+          ell += s0 + s1;
+        } else {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float w0, w1, w2, w3;
-            exp_pair(v[c * 16 + 4 * j + 0], v[c * 16 + 4 * j + 1], coef2, bias2, w0, w1);
-            exp_pair(v[c * 16 + 4 * j + 2], v[c * 16 + 4 * j + 3], coef2, bias2, w2, w3);
-            sum2 = add2(add2(sum2, f2(w0, w1)), f2(w2, w3));
-            w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
+          for (int c = 0; c < 4; ++c) {
+            uint32_t w4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              w4[j] = pack_e4m3x2(v[c * 16 + 4 * j], v[c * 16 + 4 * j + 1]) |
+                      (pack_e4m3x2(v[c * 16 + 4 * j + 2], v[c * 16 + 4 * j + 3]) << 16);
+            *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
           }
-          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          ell += kEtaP8 * (s0 + s1);  // the denominator sums the amplified fp32 weights; eta restores the unit
         }
-        float s0, s1;
-        unf2(sum2, s0, s1);
-        ell += kEtaP8 * (s0 + s1);  // the denominator sums the amplified fp32 weights; eta restores the unit
       } else {
+        // Group scales from each group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent:
+        // sigma = E4M3(448 * max w); scaled weight u = w * 2688 / sigma = 2^(x - m + log2(2688) - log2(sigma)).
+        // The four scale chains run first (interleaved), then the exponentials in batches of 32 that are all issued
+        // before any is consumed.
         uint32_t sfword = 0;
+        float bb[4], sl[4];
+        bool live[4];
 #pragma unroll
         for (int gi = 0; gi < 4; ++gi) {
-          // group scale from the group's largest weight (Eq. "v2-nvfp4-probability"), folded into the exponent:
-          // sigma = E4M3(448 * max w); scaled weight u = w * 2688 / sigma = 2^(x - m + log2(2688) - log2(sigma))
           const float gw = ex2(fmaf(gm[gi], coef, -m_new));
           const uint32_t sc = pack_e4m3x2(__fmul_rn(448.0f, gw), 0.f) & 0xffu;
           sfword |= sc << (8 * gi);
           // E4M3 code -> fp32: for normal codes the bit pattern is a shift and a re-bias; the 7 subnormal codes
           // and zero (weights below 2^-15 of the row maximum) take the general conversion
           const float sigma = sc >= 8u ? __uint_as_float((sc << 20) + 0x3C000000u) : decode_e4m3(sc);
-          const bool live = sc != 0u;
-          const float b = (live ? 11.392317422778762f - lg2(sigma) : 0.f) - m_new;  // log2(2688) = 11.3923...
-          const uint64_t bias2 = f2(b, b);
-          uint64_t sum2 = 0;
-          uint32_t c0 = 0, c1 = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float u0, u1, u2, u3;
-            exp_pair(v[gi * 16 + 4 * j + 0], v[gi * 16 + 4 * j + 1], coef2, bias2, u0, u1);
-            exp_pair(v[gi * 16 + 4 * j + 2], v[gi * 16 + 4 * j + 3], coef2, bias2, u2, u3);
-            sum2 = add2(add2(sum2, f2(u0, u1)), f2(u2, u3));
-            const uint32_t pk = pack_e2m1x4(u0, u1, u2, u3);
-            if (j < 2) c0 |= pk << (16 * j); else c1 |= pk << (16 * (j - 2));
-          }
-          // 16 keys = 8 bytes: chunk gi/2 (32 keys per 16-byte chunk), half gi&1
-          *reinterpret_cast<uint2 *>(prow + (gi >> 1) * 1024 + (gi & 1) * 8) = make_uint2(live ? c0 : 0u, live ? c1 : 0u);
-          float s0, s1;
-          unf2(sum2, s0, s1);
-          ell = fmaf(s0 + s1, live ? sigma * (1.0f / 2688.0f) : 1.0f, ell);
+          live[gi] = sc != 0u;
+          bb[gi] = (live[gi] ? 11.392317422778762f - lg2(sigma) : 0.f) - m_new;  // log2(2688) = 11.3923...
+          sl[gi] = live[gi] ? sigma * (1.0f / 2688.0f) : 1.0f;
         }
         *reinterpret_cast<uint32_t *>(smem + sm.sfp[s][g] + (r & 31) * 16 + (r >> 5) * 4) = sfword;
+        {
+          // the scores of the row become the exponent arguments, then the scaled weights, in place
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float b = bb[j >> 3];
+            unf2(fma2(f2(v[2 * j], v[2 * j + 1]), coef2, f2(b, b)), v[2 * j], v[2 * j + 1]);
+          }
+#pragma unroll
+          for (int j = 0; j < 64; ++j) v[j] = ex2(v[j]);
+#pragma unroll
+          for (int gp = 0; gp < 2; ++gp) {  // 32 keys = two groups = one 16-byte chunk of the row
+            uint32_t cw[4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const float *x = v + gp * 32 + h * 16;
+              const uint64_t sa = add2(f2(x[0], x[1]), f2(x[2], x[3])), sb = add2(f2(x[4], x[5]), f2(x[6], x[7]));
+              const uint64_t sc2 = add2(f2(x[8], x[9]), f2(x[10], x[11])), sd = add2(f2(x[12], x[13]), f2(x[14], x[15]));
+              float s0, s1;
+              unf2(add2(add2(sa, sb), add2(sc2, sd)), s0, s1);
+              ell = fmaf(s0 + s1, sl[gp * 2 + h], ell);
+              const uint32_t c0 = pack_e2m1x4(x[0], x[1], x[2], x[3]) | (pack_e2m1x4(x[4], x[5], x[6], x[7]) << 16);
+              const uint32_t c1 = pack_e2m1x4(x[8], x[9], x[10], x[11]) | (pack_e2m1x4(x[12], x[13], x[14], x[15]) << 16);
+              cw[h * 2 + 0] = live[gp * 2 + h] ? c0 : 0u;
+              cw[h * 2 + 1] = live[gp * 2 + h] ? c1 : 0u;
+            }
+            *reinterpret_cast<uint4 *>(prow + gp * 1024) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+          }
+        }
       }
       PROF_T(pt4);
       PROF_ADD(5, pt3, pt4);
