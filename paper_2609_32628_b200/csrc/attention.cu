@@ -167,14 +167,6 @@ __device__ __forceinline__ float max16(const float *x) {
   const float m3 = max3(x[9], x[10], x[11]), m4 = max3(x[12], x[13], x[14]);
   return fmaxf(max3(m0, m1, m2), max3(m3, m4, x[15]));
 }
-// exponentials of two scores: 2^(x*coef + bias) for a packed pair (one packed FMA, two ex2)
-__device__ __forceinline__ void exp_pair(float x0, float x1, uint64_t coef2, uint64_t bias2, float &w0, float &w1) {
-  float t0, t1;
-  unf2(fma2(f2(x0, x1), coef2, bias2), t0, t1);
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w0) : "f"(t0));
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(w1) : "f"(t1));
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
