@@ -265,3 +265,30 @@ def test_refresh_operands_keeps_the_selection():
     sel = [(h, a) for h in range(w1.B * w1.H) for a in range(I.R)]
     _check_attention(w2, out, mixed, sel, bad)
     assert torch.isfinite(out.float()).all()
+
+
+def test_prepare_and_attention_replay_from_a_cuda_graph():
+    """The two calls only enqueue kernels and a memset on the caller's stream (no allocation, no synchronisation), so
+    a captured graph of them replays to the same bits as the eager calls."""
+    w = SMALL["ragged64"]
+    q, k, v = _inputs(w)
+    plan, ws, out = run_gpu(w, q, k, v, zero_ws=True)
+    ws2 = torch.zeros_like(ws)
+    out2 = torch.full_like(out, float("nan"))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                      # warm-up on the capture stream (function attributes, modules)
+        da2.da2_prepare(plan, q, k, v, ws2)
+        da2.da2_attention_fwd(plan, q, k, v, ws2, out2)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        da2.da2_prepare(plan, q, k, v, ws2)
+        da2.da2_attention_fwd(plan, q, k, v, ws2, out2)
+    for _ in range(2):
+        out2.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert da2.da2_device_status(plan, ws2) == 0
+        assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
