@@ -50,7 +50,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             print(f"nvcc failed on {src}", file=sys.stderr)
     if failed:
         raise RuntimeError("building libda2.so failed")
-    subprocess.check_call([nvcc, "-shared", "-cudart", "static", "-o", LIB] + objs)
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static", "-o", LIB] + objs)
     return LIB
 
 
