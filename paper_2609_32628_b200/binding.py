@@ -204,3 +204,88 @@ def attention(plan: Plan, q, k, v, workspace=None, out=None, stream=None):
     da2_prepare(plan, q, k, v, workspace, stream)
     da2_attention_fwd(plan, q, k, v, workspace, out, stream)
     return out, workspace
+
+
+class HostPipeline:
+    """Attention on HOST tensors with the PCIe copies hidden behind the kernels.
+
+    Heads are independent problems, so the call is cut into groups of heads that flow through three CUDA streams:
+    host-to-device copies of group g+1, da2_prepare + da2_attention_fwd of group g and the device-to-host copy of
+    group g-1 run at the same time (two device slots per stage).  Everything that computes is the same C ABI; this
+    class only owns the per-group plans, buffers, streams and events.  Inputs and output must be pinned host tensors
+    for the copies to be asynchronous.
+    """
+
+    def __init__(self, B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float,
+                 frac4: float, lam: float = 0.2, rank_scope: int = DA2_RANK_ROW, groups: int = 8, device="cuda"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.BH, self.N, self.d = B * H, T * Hg * Wg, head_dim
+        groups = max(1, min(groups, self.BH))
+        base, extra = divmod(self.BH, groups)
+        self.ranges, h0 = [], 0
+        for g in range(groups):
+            n = base + (1 if g < extra else 0)
+            self.ranges.append((h0, h0 + n))
+            h0 += n
+        self.plans = {n: da2_plan(1, n, T, Hg, Wg, head_dim, frac16, frac8, frac4, lam=lam, rank_scope=rank_scope)
+                      for n in {b - a for a, b in self.ranges}}
+        nmax = max(self.plans)
+        wsb = max(int(p.info.workspace_bytes) for p in self.plans.values())
+        mk = lambda: torch.empty(nmax, self.N, self.d, dtype=torch.bfloat16, device=self.device)
+        self.slots = [dict(q=mk(), k=mk(), v=mk(), out=mk(),
+                           ws=torch.empty(wsb, dtype=torch.uint8, device=self.device)) for _ in range(2)]
+        self.s_in, self.s_c, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
+        self.launches = 0
+
+    def run(self, hq, hk, hv, hout) -> None:
+        """hq, hk, hv, hout: host bf16 [B, H, N, d] (pinned).  Returns when everything is enqueued; the caller's
+        current stream waits for the last copy."""
+        torch = self.torch
+        cur = torch.cuda.current_stream(self.device)
+        for s in (self.s_in, self.s_c, self.s_out):
+            s.wait_stream(cur)
+        fq, fk, fv, fo = (t.view(self.BH, self.N, self.d) for t in (hq, hk, hv, hout))
+        ev_c, ev_out = [], []
+        self.launches = 0
+        for gi, (a, b) in enumerate(self.ranges):
+            n, slot = b - a, self.slots[gi % 2]
+            plan = self.plans[n]
+            q, k, v, o = (slot[x][:n] for x in ("q", "k", "v", "out"))
+            with torch.cuda.stream(self.s_in):
+                if gi >= 2:
+                    self.s_in.wait_event(ev_c[gi - 2])       # the slot's previous inputs have been consumed
+                q.copy_(fq[a:b], non_blocking=True)
+                k.copy_(fk[a:b], non_blocking=True)
+                v.copy_(fv[a:b], non_blocking=True)
+                e_in = torch.cuda.Event()
+                e_in.record(self.s_in)
+            with torch.cuda.stream(self.s_c):
+                self.s_c.wait_event(e_in)
+                if gi >= 2:
+                    self.s_c.wait_event(ev_out[gi - 2])      # the slot's previous output has left the device
+                q4, k4, v4, o4 = (t.view(1, n, self.N, self.d) for t in (q, k, v, o))
+                da2_prepare(plan, q4, k4, v4, slot["ws"], self.s_c)
+                self.launches += da2_last_launch_count(plan)
+                da2_attention_fwd(plan, q4, k4, v4, slot["ws"], o4, self.s_c)
+                self.launches += da2_last_launch_count(plan)
+                e_c = torch.cuda.Event()
+                e_c.record(self.s_c)
+                ev_c.append(e_c)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(e_c)
+                fo[a:b].copy_(o, non_blocking=True)
+                e_o = torch.cuda.Event()
+                e_o.record(self.s_out)
+                ev_out.append(e_o)
+        cur.wait_stream(self.s_out)
+        cur.wait_stream(self.s_c)
+
+    def status(self) -> int:
+        """Worst device status word left in the two slots, i.e. of the last two head groups (synchronises)."""
+        worst = 0
+        for n, plan in self.plans.items():
+            for slot in self.slots:
+                worst = max(worst, da2_device_status(plan, slot["ws"]))
+        return worst

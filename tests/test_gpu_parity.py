@@ -292,3 +292,20 @@ def test_prepare_and_attention_replay_from_a_cuda_graph():
         torch.cuda.synchronize()
         assert da2.da2_device_status(plan, ws2) == 0
         assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+
+
+def test_host_pipeline_equals_the_direct_call():
+    """HostPipeline (head groups through three streams, host tensors in and out) gives the bits of one direct call."""
+    w = W("pipe", 1, 5, 64, 2, 16, 24, 0.1, 0.2, 0.3, seed=31)
+    q, k, v = _inputs(w)
+    plan, ws, out = run_gpu(w, q, k, v)
+    hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
+    for groups in (1, 2, 3, 5):   # 3 groups of 5 heads: sizes 2, 2, 1 (two plans)
+        hout = torch.full_like(hq, float("nan")).pin_memory()
+        pipe = da2.HostPipeline(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
+                                groups=groups)
+        for _ in range(2):
+            pipe.run(hq, hk, hv, hout)
+        torch.cuda.synchronize()
+        assert pipe.status() == 0
+        assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), groups
