@@ -44,7 +44,7 @@ class PlanInfo(ctypes.Structure):
                 ("off_ids", ctypes.c_uint64), ("off_select", ctypes.c_uint64), ("off_qrec", ctypes.c_uint64 * 3),
                 ("off_kvrec", ctypes.c_uint64 * 3), ("qrec_bytes", ctypes.c_uint32 * 3),
                 ("kvrec_bytes", ctypes.c_uint32 * 3), ("off_dq8", ctypes.c_uint64), ("off_dk8", ctypes.c_uint64),
-                ("off_dv8", ctypes.c_uint64)]
+                ("off_dv8", ctypes.c_uint64), ("off_order", ctypes.c_uint64)]
 
 
 def load_library():
@@ -236,6 +236,8 @@ class HostPipeline:
         mk = lambda: torch.empty(nmax, self.N, self.d, dtype=torch.bfloat16, device=self.device)
         self.slots = [dict(q=mk(), k=mk(), v=mk(), out=mk(),
                            ws=torch.empty(wsb, dtype=torch.uint8, device=self.device)) for _ in range(2)]
+        for slot in self.slots:
+            slot["ws"][:256].zero_()   # status words read as OK until a call writes them
         self.s_in, self.s_c, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
         self.launches = 0
 

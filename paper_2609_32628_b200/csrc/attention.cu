@@ -266,7 +266,9 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   const int R = p.R, pairs = (R + 1) / 2;
   const int bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
   __nv_bfloat16 *out_head = out + (size_t)bh * p.N * D;
-  const StreamInfo st0 = load_stream(p, bh, 2 * pr), st1 = load_stream(p, bh, 2 * pr + 1);
+  // the two query blocks of this CTA: equally long rows of the head (scheduling order written with the lists)
+  const uint16_t *ord = p.order + ((size_t)bh * pairs + pr) * 2;
+  const StreamInfo st0 = load_stream(p, bh, ord[0]), st1 = load_stream(p, bh, ord[1]);
 
   auto store_zero_rows = [&](int a, int first, int nthreads) {  // rows without a retained key return zero (App. C.1)
     const unsigned long long qmask = block_valid_mask(p, a);

@@ -60,6 +60,7 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
   p.counts = (int *)(w + I.off_counts);
   p.ids = (uint16_t *)(w + I.off_ids);
   p.select = (uint32_t *)(w + I.off_select);
+  p.order = (uint16_t *)(w + I.off_order);
   for (int t = 0; t < 3; ++t) {
     p.qrec[t] = w + I.off_qrec[t];
     p.kvrec[t] = w + I.off_kvrec[t];
@@ -150,6 +151,7 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   I.off_dq8 = c.take(BH * R * 4);
   I.off_dk8 = c.take(BH * R * 4);
   I.off_dv8 = c.take(BH * d * 4);
+  I.off_order = c.take(BH * (uint64_t)(2 * ((R + 1) / 2)) * 2);
   I.workspace_bytes = c.cur;
 
   const float *src[3] = {cfg->g_q, cfg->g_k, cfg->g_v};
@@ -203,6 +205,7 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
   if (select) {
     if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   }
   if (da2::launch_prep(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   plan->last_launches = launches;

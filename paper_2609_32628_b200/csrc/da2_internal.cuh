@@ -43,6 +43,7 @@ struct Params {
   uint32_t *select;         // HEAD-scope scratch
   uint8_t *qrec[3], *kvrec[3];
   float *dq8, *dk8, *dv8;
+  uint16_t *order;          // [BH][2*ceil(R/2)] query blocks by decreasing list length
 };
 
 // number of valid rows / columns of tile (ty, tx) and the 64-bit slot-valid mask of block a
@@ -70,6 +71,7 @@ cudaError_t launch_pool(const Params &p, const __nv_bfloat16 *q, const __nv_bflo
 cudaError_t launch_draft(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_map_rows(const Params &p, cudaStream_t st, int *launches);
+cudaError_t launch_order(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches);
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);

@@ -448,4 +448,39 @@ cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches) {
   return cudaGetLastError();
 }
 
+
+// Scheduling order of the query blocks of a head for the attention kernel: by decreasing list length, ties by index.
+// O(R^2) comparisons per head on lengths staged in shared memory (R is a few thousand at most).
+namespace {
+__global__ void __launch_bounds__(256) order_rows_kernel(Params p) {
+  extern __shared__ int s_len[];
+  const int bh = blockIdx.x, R = p.R, Rp = 2 * ((R + 1) / 2);
+  const int *cnt = p.counts + (size_t)bh * R * 4;
+  for (int a = threadIdx.x; a < R; a += blockDim.x) s_len[a] = cnt[a * 4] + cnt[a * 4 + 1] + cnt[a * 4 + 2];
+  __syncthreads();
+  uint16_t *ord = p.order + (size_t)bh * Rp;
+  if (threadIdx.x == 0 && Rp > R) ord[R] = 0xFFFFu;
+  for (int a = threadIdx.x; a < R; a += blockDim.x) {
+    const int la = s_len[a];
+    int pos = 0;
+    for (int b = 0; b < R; ++b) {
+      const int lb = s_len[b];
+      pos += (lb > la) || (lb == la && b < a);
+    }
+    ord[pos] = (uint16_t)a;
+  }
+}
+}  // namespace
+
+cudaError_t launch_order(const Params &p, cudaStream_t st, int *launches) {
+  const size_t smem = (size_t)p.R * sizeof(int);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(order_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  order_rows_kernel<<<p.BH, 256, smem, st>>>(p);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
 }  // namespace da2

@@ -309,3 +309,23 @@ def test_host_pipeline_equals_the_direct_call():
         torch.cuda.synchronize()
         assert pipe.status() == 0
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), groups
+
+
+@pytest.mark.parametrize("rank_scope", [0, 1])
+def test_scheduling_order_sorts_rows_by_list_length(rank_scope):
+    """The order region pairs query blocks of equal list length: a permutation of the blocks of each head, by
+    decreasing length, lower index first among equals, padded with 0xFFFF when R is odd."""
+    w = SMALL["ragged3"]
+    q, k, v = _inputs(w)
+    plan, ws, _ = run_gpu(w, q, k, v, rank_scope=rank_scope)
+    I = plan.info
+    BH, R = I.B * I.H, I.R
+    Rp = 2 * ((R + 1) // 2)
+    order = ws[I.off_order:I.off_order + BH * Rp * 2].cpu().numpy().view(np.uint16).reshape(BH, Rp)
+    counts = ws[I.off_counts:I.off_counts + BH * R * 16].cpu().numpy().view(np.int32).reshape(BH, R, 4)
+    L = counts[:, :, :3].sum(-1)
+    for h in range(BH):
+        expect = sorted(range(R), key=lambda a: (-int(L[h, a]), a))
+        assert order[h, :R].tolist() == expect
+        if Rp > R:
+            assert order[h, R] == 0xFFFF
