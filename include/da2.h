@@ -88,7 +88,8 @@ typedef struct {
   uint64_t off_dq8, off_dk8;         /* fp32[BH][R]: INT8 block scales of Q and K */
   uint64_t off_dv8;                  /* fp32[BH][d]: E4M3 per-channel scale of V */
   uint64_t off_order;                /* uint16[BH][2*ceil(R/2)]: query blocks of a head by decreasing list length
-                                        (ties: lower index first; 0xFFFF pads an odd R).  Scheduling only: the
+                                        (ties: lower index first; 0xFFFF pads an odd R), written in HEAD scope only
+                                        (per-row budgets: equal lengths, blocks 2p and 2p+1).  Scheduling only: the
                                         attention kernel gives CTA p of a head the blocks order[2p], order[2p+1],
                                         so that its two rows are equally long (the paper has no counterpart) */
 } da2_plan_info_t;

@@ -255,7 +255,9 @@ __device__ __forceinline__ StreamInfo load_stream(const Params &p, int bh, int a
   return st;
 }
 
-template <int D>
+// ORDERED: the CTA's two query blocks come from the scheduling order of the head (rows of unequal length, HEAD scope);
+// otherwise they are blocks 2p and 2p+1 (per-row budgets: every row has the same length, the order is the identity).
+template <int D, bool ORDERED>
 __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_tmem_base;
@@ -267,8 +269,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   const int bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
   __nv_bfloat16 *out_head = out + (size_t)bh * p.N * D;
   // the two query blocks of this CTA: equally long rows of the head (scheduling order written with the lists)
-  const uint16_t *ord = p.order + ((size_t)bh * pairs + pr) * 2;
-  const StreamInfo st0 = load_stream(p, bh, ord[0]), st1 = load_stream(p, bh, ord[1]);
+  int a0 = 2 * pr, a1 = 2 * pr + 1;
+  if (ORDERED) {
+    const uint16_t *ord = p.order + ((size_t)bh * pairs + pr) * 2;
+    a0 = ord[0];
+    a1 = ord[1];
+  }
+  const StreamInfo st0 = load_stream(p, bh, a0), st1 = load_stream(p, bh, a1);
 
   auto store_zero_rows = [&](int a, int first, int nthreads) {  // rows without a retained key return zero (App. C.1)
     const unsigned long long qmask = block_valid_mask(p, a);
@@ -842,15 +849,16 @@ cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t s
   const SmemMap sm = make_smem_map(p);
   cudaError_t e;
   const int grid = p.BH * ((p.R + 1) / 2);
-  if (p.d == 128) {
-    e = cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
-    if (e != cudaSuccess) return e;
-    attention_kernel<128><<<grid, NT, sm.total, st>>>(p, sm, out);
-  } else {
-    e = cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
-    if (e != cudaSuccess) return e;
-    attention_kernel<64><<<grid, NT, sm.total, st>>>(p, sm, out);
-  }
+  auto launch = [&](auto kernel) -> cudaError_t {
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, NT, sm.total, st>>>(p, sm, out);
+    return cudaSuccess;
+  };
+  const bool ordered = p.rank_scope != 0;
+  if (p.d == 128) e = ordered ? launch(attention_kernel<128, true>) : launch(attention_kernel<128, false>);
+  else e = ordered ? launch(attention_kernel<64, true>) : launch(attention_kernel<64, false>);
+  if (e != cudaSuccess) return e;
   *launches += 1;
   return cudaGetLastError();
 }

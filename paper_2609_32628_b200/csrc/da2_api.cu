@@ -205,7 +205,8 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
   if (select) {
     if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
-    if (da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    // rows of unequal length (HEAD scope) are paired by length; with per-row budgets the order is the identity
+    if (plan->info.rank_scope != 0 && da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   }
   if (da2::launch_prep(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   plan->last_launches = launches;

@@ -311,8 +311,7 @@ def test_host_pipeline_equals_the_direct_call():
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), groups
 
 
-@pytest.mark.parametrize("rank_scope", [0, 1])
-def test_scheduling_order_sorts_rows_by_list_length(rank_scope):
+def test_scheduling_order_sorts_rows_by_list_length(rank_scope=1):
     """The order region pairs query blocks of equal list length: a permutation of the blocks of each head, by
     decreasing length, lower index first among equals, padded with 0xFFFF when R is odd."""
     w = SMALL["ragged3"]
