@@ -611,3 +611,44 @@ def test_prop_3_4_bound_difference_identity():
         b2 = 2 * vmax * d2 + m8 * e8 + m4 * e4
         assert abs((b2 - b1) - (-2 * vmax * tau + (t8 * e8 + t4 * e4) / (1 - d2))) < 1e-12
         assert (b2 < b1) == (t8 * e8 + t4 * e4 < 2 * vmax * tau * (1 - d2))
+
+
+def _golden():
+    import os
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, value = line.split()[:2]
+                vals[name] = float(value)
+    return vals
+
+
+def test_golden_constants():
+    """The constants the paper prints (tests/golden/paper_constants.txt) against what the oracle computes with."""
+    g = _golden()
+    # format ranges: the largest codes decode to the printed maxima, and their product is the NVFP4 range
+    assert oracle.decode_e2m1(7) == g["e2m1_max"] and oracle.decode_e2m1(15) == -g["e2m1_max"]
+    assert oracle.decode_e4m3(0x7E) == g["e4m3_max"] and oracle.cast_e4m3(1e9) == 0x7E
+    assert g["e2m1_max"] * g["e4m3_max"] == g["nvfp4_range"]
+    # INT8: a block whose largest magnitude is `levels` gets delta = 1 + eps (to fp32) and the code `levels`
+    pl = oracle.plan(1, 8, 8)
+    x = np.zeros((1, 64, 16), np.float32)
+    x[0, 5, 3] = g["int8_levels"]
+    x[0, 6, 2] = -1.0
+    codes, delta = oracle.quant_int8(oracle.bf16_bits(torch.from_numpy(x).to(torch.bfloat16)), pl)
+    assert float(delta[0, 0]) == float(np.float32(np.float32(1.0) + np.float32(g["int8_epsilon"])))
+    assert codes.reshape(64, 16)[5, 3] == g["int8_levels"] and codes.reshape(64, 16)[6, 2] == -1
+    # E4M3 V: the per-channel scale is the channel maximum over the printed divisor
+    v = np.zeros((1, 64, 16), np.float32)
+    v[0, 9, 4] = 4.5
+    _, dc = oracle.quant_v_e4m3(oracle.bf16_bits(torch.from_numpy(v).to(torch.bfloat16)), pl)
+    assert float(dc[0, 4]) == float(np.float32(4.5) / np.float32(g["v_e4m3_divisor"])) and float(dc[0, 0]) == 0.0
+    # NVFP4: per-head scale = amax / 2688
+    assert float(oracle.nvfp4_global_scale(oracle.bf16_bits(torch.from_numpy(x).to(torch.bfloat16)))[0]) == \
+        float(np.float32(g["int8_levels"]) / np.float32(g["nvfp4_range"]))
+    # 8-bit weights: the offset amplifies a weight of 1 to just below the E4M3 maximum, and eta undoes it
+    amp = 2.0 ** g["p8_exponent_offset"]
+    assert g["e4m3_max"] - 0.2 < amp < g["e4m3_max"]
+    assert abs(g["p8_eta"] * amp - 1.0) < 5e-7
+    assert oracle.decode_e4m3(oracle.cast_e4m3(amp)) == g["e4m3_max"]
