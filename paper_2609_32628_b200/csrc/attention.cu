@@ -257,7 +257,9 @@ __device__ __forceinline__ StreamInfo load_stream(const Params &p, int bh, int a
 
 // ORDERED: the CTA's two query blocks come from the scheduling order of the head (rows of unequal length, HEAD scope);
 // otherwise they are blocks 2p and 2p+1 (per-row budgets: every row has the same length, the order is the identity).
-template <int D, bool ORDERED>
+// FP4: the plan has an NVFP4 tier.  Without one the exponentiate phase keeps the per-pair interleaved form, which is
+// the faster one for the 8-bit and bf16 bodies alone (the compiler's schedule of the unrolled softmax body decides).
+template <int D, bool ORDERED, bool FP4>
 __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_tmem_base;
@@ -633,7 +635,46 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 
       PROF_T(pt3);
       const uint64_t coef2 = f2(coef, coef);
-      if (tier != 0) {
+      if (!FP4 && tier == 2) {
+        const uint64_t bias2 = f2(-m_new, -m_new);
+        uint64_t sum2 = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint32_t w4[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float t0, t1;
+            unf2(fma2(f2(v[c * 8 + 2 * j], v[c * 8 + 2 * j + 1]), coef2, bias2), t0, t1);
+            const float w0 = ex2(t0), w1 = ex2(t1);
+            sum2 = add2(sum2, f2(w0, w1));
+            w4[j] = pack_bf16x2(w0, w1);
+          }
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+        float s0, s1;
+        unf2(sum2, s0, s1);
+        ell += s0 + s1;
+      } else if (!FP4) {
+        const uint64_t bias2 = f2(kOffsetP8 - m_new, kOffsetP8 - m_new);
+        uint64_t sum2 = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t w4[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float t0, t1, t2, t3;
+            unf2(fma2(f2(v[c * 16 + 4 * j + 0], v[c * 16 + 4 * j + 1]), coef2, bias2), t0, t1);
+            unf2(fma2(f2(v[c * 16 + 4 * j + 2], v[c * 16 + 4 * j + 3]), coef2, bias2), t2, t3);
+            const float w0 = ex2(t0), w1 = ex2(t1), w2 = ex2(t2), w3 = ex2(t3);
+            sum2 = add2(add2(sum2, f2(w0, w1)), f2(w2, w3));
+            w4[j] = pack_e4m3x2(w0, w1) | (pack_e4m3x2(w2, w3) << 16);
+          }
+          *reinterpret_cast<uint4 *>(prow + c * 1024) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+        float s0, s1;
+        unf2(sum2, s0, s1);
+        ell += kEtaP8 * (s0 + s1);  // the denominator sums the amplified fp32 weights; eta restores the unit
+      } else if (tier != 0) {
         // the scores of the row become the exponent arguments, then the weights, in place: all 64 exponentials are
         // issued before any is consumed (the 8-bit path carries the 2^8.807 offset in the exponent)
         const float b = tier == 1 ? kOffsetP8 - m_new : -m_new;
@@ -855,9 +896,14 @@ cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t s
     kernel<<<grid, NT, sm.total, st>>>(p, sm, out);
     return cudaSuccess;
   };
-  const bool ordered = p.rank_scope != 0;
-  if (p.d == 128) e = ordered ? launch(attention_kernel<128, true>) : launch(attention_kernel<128, false>);
-  else e = ordered ? launch(attention_kernel<64, true>) : launch(attention_kernel<64, false>);
+  const bool ordered = p.rank_scope != 0, fp4 = p.tier_active[0] != 0;
+  if (p.d == 128) {
+    e = ordered ? (fp4 ? launch(attention_kernel<128, true, true>) : launch(attention_kernel<128, true, false>))
+                : (fp4 ? launch(attention_kernel<128, false, true>) : launch(attention_kernel<128, false, false>));
+  } else {
+    e = ordered ? (fp4 ? launch(attention_kernel<64, true, true>) : launch(attention_kernel<64, true, false>))
+                : (fp4 ? launch(attention_kernel<64, false, true>) : launch(attention_kernel<64, false, false>));
+  }
   if (e != cudaSuccess) return e;
   *launches += 1;
   return cudaGetLastError();
