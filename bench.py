@@ -203,9 +203,9 @@ def run_da2(args, rank, world, local_rank):
 
     e2e_serial_ms = timed(serial_step)
     del dq, dk, dv
-    groups = min(8, w.B * w.H)
     pipe = da2.HostPipeline(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
-                            rank_scope=args.rank_scope, groups=groups, device=dev)
+                            rank_scope=args.rank_scope, groups="ramp", device=dev)
+    groups = [b - a for a, b in pipe.ranges]
     e2e_ms = timed(lambda: pipe.run(hq, hk, hv, hout))
     assert pipe.status() == 0, "device status after the end-to-end region"
     e2e_launches = pipe.launches
@@ -247,7 +247,7 @@ def run_da2(args, rank, world, local_rank):
                    "l2": "inputs larger than L2 (Q, K, V and operand records are several GB per step)"},
         "e2e": {"value": dense * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": out.numel() * 2,
-                "how": f"HostPipeline: {groups} groups of heads, copy-in / kernels / copy-out on three streams, "
+                "how": f"HostPipeline: groups of {groups} heads, copy-in / kernels / copy-out on three streams, "
                        f"{e2e_launches} kernels per step",
                 "serial_ms_per_step": e2e_serial_ms,
                 "serial_value": dense * world / (e2e_serial_ms * 1e-3) / 1e12},

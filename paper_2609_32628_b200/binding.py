@@ -217,16 +217,13 @@ class HostPipeline:
     """
 
     def __init__(self, B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float,
-                 frac4: float, lam: float = 0.2, rank_scope: int = DA2_RANK_ROW, groups: int = 8, device="cuda"):
+                 frac4: float, lam: float = 0.2, rank_scope: int = DA2_RANK_ROW, groups="ramp", device="cuda"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
         self.BH, self.N, self.d = B * H, T * Hg * Wg, head_dim
-        groups = max(1, min(groups, self.BH))
-        base, extra = divmod(self.BH, groups)
         self.ranges, h0 = [], 0
-        for g in range(groups):
-            n = base + (1 if g < extra else 0)
+        for n in self._group_sizes(self.BH, groups):
             self.ranges.append((h0, h0 + n))
             h0 += n
         self.plans = {n: da2_plan(1, n, T, Hg, Wg, head_dim, frac16, frac8, frac4, lam=lam, rank_scope=rank_scope)
@@ -240,6 +237,26 @@ class HostPipeline:
             slot["ws"][:256].zero_()   # status words read as OK until a call writes them
         self.s_in, self.s_c, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
         self.launches = 0
+
+    @staticmethod
+    def _group_sizes(BH: int, groups):
+        """Heads per group.  An int gives that many nearly equal groups; "ramp" gives small groups at both ends (the
+        first copy-in and the last copy-out are the only transfers that nothing hides) and large ones in between."""
+        if groups != "ramp":
+            g = max(1, min(int(groups), BH))
+            base, extra = divmod(BH, g)
+            return [base + (1 if i < extra else 0) for i in range(g)]
+        cap = max(1, -(-BH // 6))
+        up, n = [], 1
+        while n < cap and 2 * (sum(up) + n) <= BH - cap:
+            up.append(n)
+            n *= 2
+        rest = BH - 2 * sum(up)
+        mid = []
+        while rest > 0:
+            mid.append(min(cap, rest))
+            rest -= mid[-1]
+        return up + mid + up[::-1]
 
     def run(self, hq, hk, hv, hout) -> None:
         """hq, hk, hv, hout: host bf16 [B, H, N, d] (pinned).  Returns when everything is enqueued; the caller's

@@ -300,7 +300,7 @@ def test_host_pipeline_equals_the_direct_call():
     q, k, v = _inputs(w)
     plan, ws, out = run_gpu(w, q, k, v)
     hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
-    for groups in (1, 2, 3, 5):   # 3 groups of 5 heads: sizes 2, 2, 1 (two plans)
+    for groups in (1, 2, 3, 5, "ramp"):   # 3 groups of 5 heads: sizes 2, 2, 1 (two plans)
         hout = torch.full_like(hq, float("nan")).pin_memory()
         pipe = da2.HostPipeline(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
                                 groups=groups)
