@@ -565,6 +565,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       if (!PROF_WAIT(0, wait_or_abort(bar(s, B_SREADY + g), kp, abortp))) break;
       tc::fence_after_sync();
       PROF_T(pt0);
+      // the step's mask and key scale (written before its K block was requested) are read while the scores load
+      const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
+      const uint2 kmask = *reinterpret_cast<const uint2 *>(info);
+      float coef;
+      if (tier == 2) coef = c16;
+      else if (tier == 1) coef = dq8s * *reinterpret_cast<const float *>(info + 8);
+      else coef = gqk;
       float v[64];
       {
         uint32_t a0[16], a1[16], a2[16], a3[16];
@@ -596,12 +603,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       PROF_ADD(3, pt0, pt1);
       tc::fence_before_sync();
       warp_arrive(bar(s, B_SFREE + g));
-      const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
-      const uint2 kmask = *reinterpret_cast<const uint2 *>(info);
-      float coef;
-      if (tier == 2) coef = c16;
-      else if (tier == 1) coef = dq8s * *reinterpret_cast<const float *>(info + 8);
-      else coef = gqk;
       if ((kmask.x & kmask.y) != 0xffffffffu) {  // ragged edge tile: padding keys take no part
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
