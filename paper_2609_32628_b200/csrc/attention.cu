@@ -8,15 +8,17 @@
 //
 // Mapping onto sm_100a
 //   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 576 threads in five roles:
-//     warps 0-7   softmax: stream = (warp%4)/2, two threads per query row (32 of the 64 key columns each); they read
-//                 S from TMEM, keep h and a partial l, and write P~ (and its NVFP4 scale factors) to shared memory
+//     warps 0-7   softmax: stream = (warp%4)/2; warps w and w+4 own the same 32 query rows and take alternate steps,
+//                 one thread per 64-key row; they read S from TMEM, keep h and a partial l, and write P~ (and its
+//                 NVFP4 scale factors) to shared memory
 //     warps 8-11  correction + epilogue: rescale the accumulator columns of queries whose maximum moved, apply the
 //                 per-channel unit change at a segment boundary, and finally normalise, transpose and store
 //     warps 12,13 S = Q K^T issue, one warp per stream (tcgen05.mma, accumulators in TMEM), two steps ahead
 //     warps 14,15 O^T += V^T P~^T issue, one warp per stream.  The issuing warps' instruction counts are on the
 //                 critical path of every step: their loops are warp-uniform (one elected lane issues), operand
 //                 descriptors are built once and only offset inside the loop
-//     warps 16,17 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings
+//     warps 16,17 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings; a
+//                 warp-uniform loop in which lane l holds list entry 32*batch + l (address, mask, key scale)
 //   S   = Q K^T   : M = 128, N = 64 keys, K = d.  The block-scaled instruction only exists at M = 128, so stream 0's
 //                   queries sit in rows 0..63 and stream 1's in rows 64..127 (its operand descriptor starts 1 KB
 //                   early); the other 64 rows of each product are don't-care.  S is double buffered.
@@ -25,10 +27,12 @@
 //                   per-channel unit changes (eta*delta_c^V, g_V/2688) per-lane scalars.
 //   kinds         : kind::f16 (BF16); kind::i8 for QK^T + kind::f8f6f4 E4M3 x E4M3 for PV (App. C.1); and
 //                   kind::mxf4nvf4 with E4M3 scales per 16 elements (NVFP4), scale factors moved by tcgen05.cp.
-// The softmax is the bound (one ex2 per score on a 16-lane/clk unit), so its inner loops are written to spend as few
-// issue slots per score as possible: the row maximum is taken on raw accumulator values, the scale and the maximum
-// are folded into one FMA feeding ex2, int32 scores become floats through a magic-number add folded into that FMA,
-// and the NVFP4 group scale is folded into the exponent so the scaled weight needs no extra multiply.
+// The softmax sets the pace (one ex2 per score on a 16-lane/clk unit, and a chain of hand-offs per step): the row
+// maximum is taken on raw accumulator values, the scale and the maximum are folded into one FMA feeding ex2, int32
+// scores become floats through a magic-number add, the NVFP4 group scale is folded into the exponent so the scaled
+// weight needs no extra multiply, and the exponentiate phase runs over the whole row in batches (all arguments, all
+// exponentials, then sums and packing), which gives the single warp the instruction-level parallelism it lacks when
+// the three are interleaved per pair.
 // Every wait on an mbarrier is bounded; a wait that gives up records device status "timeout", all roles leave their
 // loops and the CTA exits normally after releasing TMEM.
 #include <cuda_fp8.h>
