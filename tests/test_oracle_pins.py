@@ -596,6 +596,68 @@ def test_reconstruction_identity_and_error_bound(mix):
         assert (rel[t[kept] == 16] <= 2.0 ** -8).all()
         big8 = (t[kept] == 8) & (dbg["what"][kept] > 0.0022326917 * 2.0 ** -6)
         assert (rel[big8] <= 2.0 ** -4 + 1e-3).all()
+        # NVFP4 weights: the error is at most half the widest E2M1 gap in units of the group scale, i.e. about a
+        # sixth of the largest weight of the row's block at the time it was processed (<= 1)
+        assert (np.abs(dbg["what"] - np.where(kept, np.exp(np.where(kept, dbg["shat"] - dbg["h_at"], 0)), 0.0))[kept][t[kept] == 4]
+                <= (1 + 2.0 ** -3) / 6.0).all()
+
+
+
+_E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def _e2m1_nearest_even(x: float) -> float:
+    """Nearest E2M1 magnitude by exhaustive search; a tie goes to the neighbour with the even code."""
+    dist = np.abs(_E2M1_VALUES - x)
+    best = np.flatnonzero(dist == dist.min())
+    if len(best) == 2:
+        return float(_E2M1_VALUES[best[0] if best[0] % 2 == 0 else best[1]])
+    return float(_E2M1_VALUES[best[0]])
+
+
+@pytest.mark.parametrize("grid,mix", [((1, 12, 20), (4, 1, 1)), ((2, 16, 16), (6, 0, 0)), ((1, 9, 17), (3, 2, 0))])
+def test_online_nvfp4_weight_quantiser_is_the_printed_formula(grid, mix):
+    """Eq. 'v2-nvfp4-probability' on non-uniform weights, rebuilt outside the oracle: groups are the 16 consecutive
+    key slots 16g..16g+15 of a block (padding counts as 0), sigma_P = E4M3(448 max_G w) through torch's
+    float8_e4m3fn cast, the code is the nearest E2M1 value of 2688 w / sigma_P (ties to the even code, by search),
+    and the weight the numerator uses is sigma_P / 2688 times that value; a zero scale zeroes the group."""
+    rng = np.random.default_rng(23)
+    d = 32
+    pl, q, k, v = _setup(rng, *grid, d, scale_q=2.5)
+    ops = oracle.quantize_all(bits(q), bits(k), bits(v), pl)
+    s = 1 / math.sqrt(d)
+    ids, counts = _mixed_lists(rng, 1, pl.R, *mix)
+    n_checked = n_zero_groups = n_nonuniform = 0
+    for (a, ju) in ((0, 0), (pl.R - 1, 0), (1, 9)):
+        if pl.slot_token[a, ju] < 0:
+            continue
+        dbg = oracle.attention_row_debug(bits(q), bits(k), bits(v), pl, ids, counts, ops, s, 0, a, ju)
+        for b in ids[0, a, :mix[0]]:
+            for g in range(4):
+                toks = pl.slot_token[b, 16 * g:16 * g + 16]
+                valid = toks >= 0
+                if not valid.any():
+                    continue
+                tv = toks[valid]
+                assert (dbg["tier"][tv] == 4).all()
+                w = np.zeros(16, np.float32)
+                w[valid] = np.exp(dbg["shat"][tv] - dbg["h_at"][tv]).astype(np.float32)
+                gm = np.float32(w.max())
+                sigma = float(torch.tensor([np.float32(448.0) * gm], dtype=torch.float32)
+                              .to(torch.float8_e4m3fn).to(torch.float32)[0])
+                expect = np.zeros(16)
+                if sigma > 0.0:
+                    for i in range(16):
+                        r = np.float32(2688.0 * float(w[i]) / sigma)
+                        expect[i] = sigma / 2688.0 * _e2m1_nearest_even(float(r))
+                else:
+                    n_zero_groups += 1
+                assert np.array_equal(dbg["what"][tv], expect[valid]), (a, ju, b, g)
+                # coarse bound of the format: half of the widest E2M1 gap (4..6) in units of sigma_P/2688 ~ max/6
+                assert (np.abs(expect[valid] - w[valid]) <= float(gm) / 6.0 * (1 + 2.0 ** -3) + 1e-30).all()
+                n_checked += int(valid.sum())
+                n_nonuniform += int(len(np.unique(expect[valid])) > 1)
+    assert n_checked > 200 and n_nonuniform > 10
 
 
 def test_prop_3_4_bound_difference_identity():
