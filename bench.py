@@ -100,8 +100,115 @@ def flop_counts(w, plan, ws):
                 valid[t] = float((keys * nv[None, :]).sum().item()) * 4 * d
             lo += n
     else:
-        valid = list(padded)
+        # head-level budget: rows of unequal length; entry e of row a sits at ids[head][offset_a + e]
+        per_head = int(I.ids_per_head)
+        ids_all = (ws[I.off_ids:I.off_ids + BH * per_head * 2].view(torch.int16).view(BH, per_head).long()) & 0xffff
+        rows = torch.arange(R, device=ws.device)
+        for h in range(BH):
+            n3, off = cnt[h, :, :3], cnt[h, :, 3]
+            n = n3.sum(-1)
+            total = int(n.sum().item())
+            if total == 0:
+                continue
+            row_of = torch.repeat_interleave(rows, n)
+            start = torch.repeat_interleave(torch.cumsum(n, 0) - n, n)
+            within = torch.arange(total, device=ws.device) - start
+            key = ids_all[h, torch.repeat_interleave(off, n) + within]
+            tier = (within >= torch.repeat_interleave(n3[:, 0], n)).long() + \
+                   (within >= torch.repeat_interleave(n3[:, 0] + n3[:, 1], n)).long()
+            pair = nv[row_of] * nv[key]
+            for t in range(3):
+                valid[t] += float(pair[tier == t].sum().item()) * 4 * d
     return dense, padded, valid
+
+
+MMA_KINDS = ("bf16", "int8", "e4m3", "nvfp4")
+MMA_K = (16, 32, 32, 64)
+
+
+def mma_peaks(iters: int = 4000):
+    """tcgen05.mma microbenchmark on every SM: TFLOP/s and cycles per instruction per kind at M = 128 and
+    N = 64, 128, 256 (operands in shared memory)."""
+    import paper_2609_32628_b200 as da2
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    out = torch.zeros(4, dtype=torch.int64, device=dev)
+    rows = []
+    for kind, name in enumerate(MMA_KINDS):
+        for n in (64, 128, 256):
+            for _ in range(2):
+                da2.da2_tcgen05_peak(kind, n, iters, sms, out)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            da2.da2_tcgen05_peak(kind, n, iters, sms, out)
+            e1.record()
+            torch.cuda.synchronize()
+            cyc, instr, fail = (int(x) for x in out[:3].tolist())
+            assert fail == 0, "the microbenchmark's bounded wait gave up"
+            ms = e0.elapsed_time(e1)
+            flops = 2.0 * 128 * n * MMA_K[kind] * instr * sms
+            rows.append({"kind": name, "n": n, "tflops": flops / (ms * 1e-3) / 1e12, "cycles_per_mma": cyc / instr,
+                         "ms": ms})
+    return {"sms": sms, "iters": iters, "rows": rows}
+
+
+def sweep(steps: int = 5, warmup: int = 3):
+    """The budget sweep: five grids (8k to 131k tokens, 24 heads, d = 128) x high tier {0, 5, 10, 20} % (8-bit) x low
+    tier {0, 20, 40, 60} % (NVFP4) without the empty 0/0 point, plus the two dense endpoints (every block 8-bit, every
+    block bf16) per grid.  Each point is timed as a full call (da2_prepare + da2_attention_fwd), one JSON line each."""
+    import paper_2609_32628_b200 as da2
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    for gi in range(len(da2_inputs.SWEEP_GRIDS)):
+        points = [(h, l, False) for h in (0.0, 0.05, 0.10, 0.20) for l in (0.0, 0.20, 0.40, 0.60) if h + l > 0]
+        points += [(1.0, 0.0, False), (1.0, 0.0, True)]
+        base = da2_inputs.sweep_workload(gi, 0.05, 0.20)
+        q, k, v = da2_inputs.make_qkv(base, dev)
+        out = torch.empty_like(q)
+        for high, low, bf16 in points:
+            w = da2_inputs.sweep_workload(gi, high, low, high_is_bf16=bf16)
+            plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam)
+            ws = torch.empty(int(plan.info.workspace_bytes), dtype=torch.uint8, device=dev)
+            for _ in range(warmup):
+                da2.da2_prepare(plan, q, k, v, ws)
+                da2.da2_attention_fwd(plan, q, k, v, ws, out)
+            torch.cuda.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+            ev[0].record()
+            for i in range(steps):
+                da2.da2_prepare(plan, q, k, v, ws)
+                ev[2 * i + 1].record()
+                da2.da2_attention_fwd(plan, q, k, v, ws, out)
+                ev[2 * i + 2].record()
+            torch.cuda.synchronize()
+            assert da2.da2_device_status(plan, ws) == 0
+            ms = ev[0].elapsed_time(ev[-1]) / steps
+            attn = float(np.mean([ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(steps)]))
+            dense, padded, valid = flop_counts(w, plan, ws)
+            t_roof = sum(valid[t] / (peaks["bf16"] * 1e12 * NOMINAL_RATIO[t]) for t in range(3)) * 1e3
+            print(json.dumps({"grid": [w.T, w.Hg, w.Wg], "tokens": w.N, "high": high, "low": low,
+                              "high_tier": "bf16" if bf16 else "8-bit", "ms_call": ms, "ms_attention": attn,
+                              "dense_equiv_tflops": dense / (ms * 1e-3) / 1e12,
+                              "frac_of_measured_roofline": t_roof / attn if attn > 0 else None}), flush=True)
+            del ws, plan
+        del q, k, v, out
+        torch.cuda.empty_cache()
+
+
+def microbench_peaks():
+    """Per-kind tensor peaks (TFLOP/s, best N) from the committed microbenchmark summary, or None."""
+    path = os.path.join(ROOT, "profiles", "tcgen05_mma_peaks.md")
+    if not os.path.exists(path):
+        return None
+    best = {}
+    for ln in open(path):
+        if ln.startswith("kind="):
+            f = dict(x.split("=") for x in ln.split())
+            best[f["kind"]] = max(best.get(f["kind"], 0.0), float(f["tflops"]))
+    return best or None
 
 
 def rank_workload(name: str, rank: int):
@@ -234,8 +341,18 @@ def run_da2(args, rank, world, local_rank):
         "flops_valid": {"nvfp4": valid[0], "int8_e4m3": valid[1], "bf16": valid[2]},
         "flops_padded": {"nvfp4": padded[0], "int8_e4m3": padded[1], "bf16": padded[2]},
         "frac_of_nominal_padded": t_roof_nominal_ms / attn_ms if attn_ms > 0 else None,
+        "frac_of_nominal_valid": sum(valid[t] / (2.25e15 * NOMINAL_RATIO[t]) for t in range(3)) * 1e3 / attn_ms
+                                 if attn_ms > 0 else None,
         "ms_prepare": prep_ms,
     }
+    mb = microbench_peaks()
+    if mb and attn_ms > 0:
+        # this GPU's own tcgen05 peaks per kind (best tile shape of the committed microbenchmark); the 8-bit tier is
+        # half INT8 (scores) and half E4M3 (values)
+        t_mb = (valid[0] / (mb["nvfp4"] * 1e12) + valid[1] * 0.5 / (mb["int8"] * 1e12) +
+                valid[1] * 0.5 / (mb["e4m3"] * 1e12) + valid[2] / (mb["bf16"] * 1e12)) * 1e3
+        roofline["frac_of_microbenchmark_peaks"] = t_mb / attn_ms
+        roofline["microbenchmark_peaks_tflops"] = mb
     line = {
         "metric": METRIC, "value": dense * world / (ms_per_step * 1e-3) / 1e12, "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -323,7 +440,29 @@ def main():
     ap.add_argument("--rank-scope", type=int, default=0, choices=[0, 1])
     ap.add_argument("--cpu-blocks", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mma-peaks", action="store_true",
+                    help="run the tcgen05.mma microbenchmark (per-kind tensor peaks) instead of the benchmark")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every point of the budget sweep (one JSON line per point) instead of the benchmark")
     args = ap.parse_args()
+    if args.sweep:
+        sweep(args.steps, max(3, args.warmup))
+        return
+    if args.mma_peaks:
+        res = mma_peaks()
+        for r in res["rows"]:
+            print(f"kind={r['kind']} n={r['n']} tflops={r['tflops']:.1f} cycles_per_mma={r['cycles_per_mma']:.1f}")
+        print(json.dumps(res))
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "da2":
+        # started as a plain script: launch the N ranks (one process per GPU) and let rank 0 print the line
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

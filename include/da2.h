@@ -12,13 +12,17 @@
  *   - q, k, v, out: DEVICE pointers, contiguous bf16 [B, H, N, head_dim], N = T*Hg*Wg, raster token order
  *     u = (t*Hg + y)*Wg + x, 16-byte aligned.  out must not alias the inputs.
  *   - workspace: DEVICE pointer, 256-byte aligned, at least da2_plan_info().workspace_bytes long.  The caller owns
- *     all device memory; the library allocates none and keeps no device state between calls.
+ *     all device memory; the library allocates none and keeps no device state between calls (one exception:
+ *     da2_draft_map_noalloc, which owns a fixed scratch array, see there).
  *   - stream: a cudaStream_t passed as void* (NULL = default stream).  da2_prepare and da2_attention_fwd only
  *     enqueue work and never synchronise.
  *   - Errors are return codes.  Argument errors are detected before any launch.  A device-side bounded wait that
  *     gives up records a code in the workspace status word; da2_device_status reports it.
- *   - The plan is host memory owned by the library until da2_plan_destroy; it is immutable and may be reused for
- *     any number of calls with the same shapes and budgets (the partition is reused across layers and steps).
+ *   - The plan is host memory owned by the library until da2_plan_destroy; it is immutable (no call writes to it,
+ *     so threads may share one) and may be reused for any number of calls with the same shapes and budgets (the
+ *     partition is reused across layers and steps).
+ *   - Limits: B*H <= 32767 and R = T*ceil(Hg/8)*ceil(Wg/8) <= 16384; beyond them da2_plan returns
+ *     DA2_ERR_UNSUPPORTED.
  */
 #ifndef DA2_H_
 #define DA2_H_
@@ -139,8 +143,24 @@ da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void
 /* Synchronises stream, reads the workspace status word; DA2_OK, DA2_ERR_TIMEOUT or DA2_ERR_INTERNAL. */
 da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, void *stream);
 
-/* Number of kernels the last da2_prepare / da2_attention_fwd call on this plan enqueued (for launch accounting). */
+/* Number of kernels that the CALLING THREAD's last da2_prepare / da2_refresh_operands / da2_attention_fwd enqueued
+ * (launch accounting; kept per thread, so the plan stays immutable).  plan must be non-NULL. */
 int32_t da2_last_launch_count(const da2_plan_t *plan);
+
+/* Failure-path probe (the paper has no counterpart; it exists so that the bounded device-side waits can be tested
+ * without faulting or hanging a GPU).  Enqueues one small kernel that waits, through the same bounded wait the
+ * attention kernel uses, on a barrier that nothing ever completes; after limit_cycles GPU clock cycles
+ * (1 .. 2e9) the wait gives up, the kernel writes the time-out code into the workspace status word and returns
+ * normally.  da2_device_status then reports DA2_ERR_TIMEOUT; the next da2_prepare clears the word. */
+da2_status_t da2_probe_bounded_wait(const da2_plan_t *plan, void *workspace, int64_t limit_cycles, void *stream);
+
+/* Tensor-core microbenchmark (diagnostic; the paper has no counterpart).  Every one of `ctas` CTAs issues
+ * 4*iters back-to-back tcgen05.mma instructions of one kind with M = 128 and the given N (64, 128 or 256), operands
+ * in shared memory, accumulators in tensor memory.  kind: 0 bf16 (K = 16 per instruction), 1 INT8 (K = 32),
+ * 2 E4M3 (K = 32), 3 block-scaled NVFP4 (K = 64).  out_dev: DEVICE int64[4]: [0] clock cycles CTA 0 needed,
+ * [1] instructions it issued, [2] non-zero if its bounded wait for completion gave up.  Flops per instruction are
+ * 2*128*N*K.  Enqueues on stream; time the launch with events for a whole-GPU figure. */
+da2_status_t da2_tcgen05_peak(int32_t kind, int32_t n, int32_t iters, int32_t ctas, void *out_dev, void *stream);
 
 /*
  * Draft attention map without any device allocation or caller workspace (the paper has no counterpart: this is a
@@ -154,7 +174,8 @@ int32_t da2_last_launch_count(const da2_plan_t *plan);
  *   q_avg, q_max, k_avg, k_max : DEVICE, fp32 [BH][R][head_dim], 16-byte aligned (region descriptors, inputs)
  *   map_out                    : DEVICE, fp32 [BH][R][R] (output, rows sum to 1)
  *   limit                      : BH*R*R <= 1,048,576 and R <= 16384, head_dim a multiple of 16; larger problems
- *                                return DA2_ERR_WORKSPACE_TOO_SMALL and launch nothing
+ *                                return DA2_ERR_WORKSPACE_TOO_SMALL and launch nothing.  BH <= 32767 (a launch
+ *                                dimension): more heads return DA2_ERR_UNSUPPORTED and launch nothing
  * The first call on each device looks up the array's device address (with that device current); make that first
  * call outside any stream capture.  All calls on a device share the array, which keeps the previous call's
  * contents; every entry a call reads is written by that call first, so nothing needs clearing, but two calls whose

@@ -70,6 +70,8 @@ def load_library():
         lib.da2_device_status.argtypes = [vp, vp, vp]
         lib.da2_last_launch_count.restype = ctypes.c_int32
         lib.da2_last_launch_count.argtypes = [vp]
+        lib.da2_probe_bounded_wait.restype = ctypes.c_int
+        lib.da2_probe_bounded_wait.argtypes = [vp, vp, ctypes.c_int64, vp]
         lib.da2_plan_destroy.restype = None
         lib.da2_plan_destroy.argtypes = [vp]
         lib.da2_status_string.restype = ctypes.c_char_p
@@ -165,6 +167,25 @@ def da2_device_status(plan: Plan, workspace, stream=None) -> int:
     return int(load_library().da2_device_status(plan.handle, _ptr(workspace), _stream(stream)))
 
 
+def da2_probe_bounded_wait(plan: Plan, workspace, limit_cycles: int, stream=None) -> None:
+    """Failure-path probe: one kernel whose bounded wait runs out after limit_cycles; da2_device_status then reports
+    DA2_ERR_TIMEOUT (5) for this workspace."""
+    rc = load_library().da2_probe_bounded_wait(plan.handle, _ptr(workspace), int(limit_cycles), _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_probe_bounded_wait")
+
+
+def da2_tcgen05_peak(kind: int, n: int, iters: int, ctas: int, out_dev, stream=None) -> None:
+    """Tensor-core microbenchmark launch (see include/da2.h); out_dev: CUDA int64[4]."""
+    lib = load_library()
+    fn = lib.da2_tcgen05_peak
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+    rc = fn(kind, n, iters, ctas, _ptr(out_dev), _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_tcgen05_peak")
+
+
 def da2_last_launch_count(plan: Plan) -> int:
     return int(load_library().da2_last_launch_count(plan.handle))
 
@@ -237,6 +258,9 @@ class HostPipeline:
             slot["ws"][:256].zero_()   # status words read as OK until a call writes them
         self.s_in, self.s_c, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
         self.launches = 0
+        # one status word per head group, copied out after the group's kernels: the next group that reuses the slot
+        # clears the slot's word, so the slots alone would only remember the last two groups
+        self.group_status = torch.zeros(len(self.ranges), 4, dtype=torch.int32).pin_memory()
 
     @staticmethod
     def _group_sizes(BH: int, groups):
@@ -289,6 +313,8 @@ class HostPipeline:
                 self.launches += da2_last_launch_count(plan)
                 da2_attention_fwd(plan, q4, k4, v4, slot["ws"], o4, self.s_c)
                 self.launches += da2_last_launch_count(plan)
+                off = int(plan.info.off_status)
+                self.group_status[gi].copy_(slot["ws"][off:off + 16].view(torch.int32), non_blocking=True)
                 e_c = torch.cuda.Event()
                 e_c.record(self.s_c)
                 ev_c.append(e_c)
@@ -302,9 +328,10 @@ class HostPipeline:
         cur.wait_stream(self.s_c)
 
     def status(self) -> int:
-        """Worst device status word left in the two slots, i.e. of the last two head groups (synchronises)."""
+        """Worst device status over all head groups of the last run (synchronises): 0 = DA2_OK, 5 = DA2_ERR_TIMEOUT
+        (a bounded wait gave up), 6 = DA2_ERR_INTERNAL (e.g. a list id out of range)."""
+        self.torch.cuda.synchronize(self.device)
         worst = 0
-        for n, plan in self.plans.items():
-            for slot in self.slots:
-                worst = max(worst, da2_device_status(plan, slot["ws"]))
+        for word in self.group_status[:, 0].tolist():
+            worst = max(worst, 0 if word == 0 else (5 if word == 1 else 6))
         return worst

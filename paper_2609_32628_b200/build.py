@@ -34,10 +34,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
                "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
-        if os.environ.get("DA2_PROF"):
-            cmd.insert(1, "-DDA2_PROF")
-        for flag in os.environ.get("DA2_NVCC_FLAGS", "").split():
-            cmd.insert(1, flag)
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False

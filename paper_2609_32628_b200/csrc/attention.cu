@@ -202,34 +202,25 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
 // in hardware for a while before it reports failure, so the retry loop issues few instructions (the variant with an
 // explicit time hint is expanded into a polling loop with nanosleep and clock reads: more instructions, same run
 // time).  The bound is on elapsed clock cycles, checked once per 16 tries.
-__device__ __forceinline__ bool wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+constexpr long long kWaitLimitCycles = 400000000ll;  // about 0.2 s
+__device__ __forceinline__ bool wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit = kWaitLimitCycles) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int k = 0; k < 16; ++k)
       if (tc::mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > 400000000ll) break;  // about 0.2 s
+    if (clock64() - t0 > limit) break;
   }
   atomicCAS(const_cast<int *>(abort_flag), 0, 1 + (int)(tc::smem_u32(bar) & 0xffff));
   return false;
 }
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                              long long limit = kWaitLimitCycles) {
   if (tc::mbar_try_wait(bar, parity)) return true;
-  return wait_slow(bar, parity, abort_flag);
+  return wait_slow(bar, parity, abort_flag, limit);
 }
-
-#ifdef DA2_PROF
-// Profiling build only: cycles spent in each wait site of one CTA, accumulated into the status words.
-#define PROF_WAIT(site, call) ([&]() { const long long t_ = clock64(); const bool ok_ = (call); \
-                                       prof_acc[site] += clock64() - t_; return ok_; }())
-#define PROF_T(var) const long long var = clock64()
-#define PROF_ADD(site, a, b) prof_acc[site] += (b) - (a)
-#else
-#define PROF_WAIT(site, call) (call)
-#define PROF_T(var)
-#define PROF_ADD(site, a, b)
-#endif
 
 // One arrival per warp: every lane's earlier writes are ordered before the elected lane's arrive by the warp barrier.
 // (A per-thread arrive is a shared-memory atomic per thread; hundreds of them per step dominate the step time.)
@@ -335,10 +326,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   tc::fence_after_sync();
   const uint32_t tmem = s_tmem_base;
   volatile int *abortp = &s_abort;
-#ifdef DA2_PROF
-  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  const long long prof_t0 = clock64();
-#endif
 
   // =========================================================================================== loader warps
   if (warp >= kLoadWarp0) {
@@ -400,7 +387,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         const uint8_t *rec = reinterpret_cast<const uint8_t *>(((unsigned long long)rhi << 32) | rlo);
         const uint32_t kb = i < S.n4 ? kb0 : (i < S.n48 ? kb1 : kb2);
         const uint32_t vb = i < S.n4 ? vb0 : (i < S.n48 ? vb1 : vb2);
-        if (kwrapped && !PROF_WAIT(0, wait_or_abort(bar(s, B_KFREE + kk), kpar, abortp))) break;
+        if (kwrapped && !wait_or_abort(bar(s, B_KFREE + kk), kpar, abortp)) break;
         if (tc::elect_one()) {
           // the step's mask and key scale enter the info ring before the data the softmax waits for is requested
           *reinterpret_cast<uint4 *>(s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16) =
@@ -409,7 +396,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           tc::bulk_g2s(kdst + kk * sm.kstage, rec, kb, bar(s, B_FULLK + kk));
         }
         __syncwarp();
-        if (vwrapped && !PROF_WAIT(1, wait_or_abort(bar(s, B_VFREE + vv), vpar, abortp))) break;
+        if (vwrapped && !wait_or_abort(bar(s, B_VFREE + vv), vpar, abortp)) break;
         if (tc::elect_one()) {
           tc::mbar_arrive_expect_tx(bar(s, B_FULLV + vv), vb);
           tc::bulk_g2s(vdst + vv * sm.vstage, rec + kb, vb, bar(s, B_FULLV + vv));
@@ -462,10 +449,9 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       // the score tiles are double buffered, so Q K^T runs up to two steps ahead of the softmax
       for (int j = 0; j < S.L; ++j) {
         const int g = j & 1;
-        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp))) break;
-        if (!PROF_WAIT(1, wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp))) break;
+        if (!wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp)) break;
+        if (!wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp)) break;
         tc::fence_after_sync();
-        PROF_T(mq0);
         const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
         const uint32_t d_s = tmem + col_s(s, g);
         if (tc::elect_one()) {
@@ -487,8 +473,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           tc::mma_commit(bar(s, B_KFREE + kk));
         }
         __syncwarp();
-        PROF_T(mq1);
-        PROF_ADD(5, mq0, mq1);
         if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
       }
     }
@@ -514,10 +498,9 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       for (int j = 0; j < S.L; ++j) {
         // ---- O^T += V(j)^T P(j)^T, once P(j) is written and the accumulator is rescaled for step j
         const int g = j & 1;
-        if (!PROF_WAIT(2, wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp))) break;
-        if (!PROF_WAIT(3, wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp))) break;
+        if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
+        if (!wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp)) break;
         tc::fence_after_sync();
-        PROF_T(mp0);
         const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
         const uint32_t acc = j > 0;
         if (tc::elect_one()) {
@@ -538,8 +521,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           tc::mma_commit(bar(s, B_VFREE + vv));
         }
         __syncwarp();
-        PROF_T(mp1);
-        PROF_ADD(6, mp0, mp1);
         if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
       }
     }
@@ -566,9 +547,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     for (int i = par; i < S.L; i += 2) {
       const int tier = S.tier(i);
       const uint32_t kp = (uint32_t)(i >> 1) & 1u;  // completion parity of this parity's k-th step
-      if (!PROF_WAIT(0, wait_or_abort(bar(s, B_SREADY + g), kp, abortp))) break;
+      if (!wait_or_abort(bar(s, B_SREADY + g), kp, abortp)) break;
       tc::fence_after_sync();
-      PROF_T(pt0);
       // the step's mask and key scale (written before its K block was requested) are read while the scores load
       const uint8_t *info = s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16;
       const uint2 kmask = *reinterpret_cast<const uint2 *>(info);
@@ -603,8 +583,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           }
         }
       }
-      PROF_T(pt1);
-      PROF_ADD(3, pt0, pt1);
       tc::fence_before_sync();
       warp_arrive(bar(s, B_SFREE + g));
       if ((kmask.x & kmask.y) != 0xffffffffu) {  // ragged edge tile: padding keys take no part
@@ -619,14 +597,12 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 #pragma unroll
       for (int q = 0; q < 4; ++q) gm[q] = max16(v + q * 16);
       const float pmax = fmaxf(max3(gm[0], gm[1], gm[2]), gm[3]) * coef;  // log2 domain
-      PROF_T(pt2);
-      PROF_ADD(4, pt1, pt2);
       // PV(i-2) done: this parity's P buffer is free and the correction warps are past step i-2
-      if (i >= 2 && !PROF_WAIT(1, wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp))) break;
+      if (i >= 2 && !wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp)) break;
       // running maximum after step i-1, published by the other warp
       float h_prev = -INFINITY;
       if (i > 0) {
-        if (!PROF_WAIT(2, wait_or_abort(bar(s, B_XREADY + (g ^ 1)), (uint32_t)((i - 1) >> 1) & 1u, abortp))) break;
+        if (!wait_or_abort(bar(s, B_XREADY + (g ^ 1)), (uint32_t)((i - 1) >> 1) & 1u, abortp)) break;
         h_prev = *other_h;
       }
       const float m_new = fmaxf(h_prev, pmax);
@@ -638,7 +614,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       ell *= ex2(h_own - m_new);
       h_own = m_new;
 
-      PROF_T(pt3);
       const uint64_t coef2 = f2(coef, coef);
       if (!FP4 && tier == 2) {
         const uint64_t bias2 = f2(-m_new, -m_new);
@@ -762,12 +737,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
           }
         }
       }
-      PROF_T(pt4);
-      PROF_ADD(5, pt3, pt4);
       tc::fence_async_smem();
       warp_arrive(bar(s, B_PREADY + g));
-      PROF_T(pt5);
-      PROF_ADD(6, pt4, pt5);
     }
     if (S.L > 0) {
       s_ell[(s * 2 + par) * 64 + r] = ell;
@@ -793,13 +764,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         const StreamInfo &S = s ? st1 : st0;
         if (i >= S.L || dead) continue;
         const int g = i & 1;
-        if (!PROF_WAIT(0, wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp))) { dead = true; continue; }
+        if (!wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp)) { dead = true; continue; }
         if (i > 0) {
           const int tier = S.tier(i);
           const bool tier_switch = (i == S.n4) || (i == S.n48);
           const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * 2 + g) * 2);
           if ((moved.x | moved.y) != 0u || tier_switch) {
-            if (!PROF_WAIT(1, wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp))) { dead = true; continue; }
+            if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp)) { dead = true; continue; }
             tc::fence_after_sync();
             float lane_factor = 1.0f;
             if (tier_switch && ch < D) {
@@ -871,15 +842,6 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     }
   }
 
-#ifdef DA2_PROF
-  if (blockIdx.x == gridDim.x / 2 && lane == 0) {
-    const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == 8 ? 2 : warp == 12 ? 3 : warp == 16 ? 4 : warp == 14 ? 5 : -1;
-    if (role >= 0) {
-      prof_acc[7] = clock64() - prof_t0;
-      for (int k = 0; k < 8; ++k) p.status[8 + role * 8 + k] = (int)(prof_acc[k] >> 4);  // units of 16 cycles
-    }
-  }
-#endif
   tc::fence_before_sync();
   __syncthreads();
   if (s_abort && tid == 0) {
@@ -889,7 +851,33 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   if (warp == 0) tc::tmem_dealloc(tmem, kTmemCols);
 }
 
+// Failure-path probe: one warp waits, through the very wait the attention kernel uses, on an mbarrier that nothing
+// ever completes.  The wait gives up after `limit` cycles, the kernel records the same status the attention kernel
+// would (timeout + the barrier's offset) and returns normally: no trap, no endless loop, the context stays usable.
+__global__ void bounded_wait_probe_kernel(int *status, long long limit) {
+  __shared__ uint64_t never;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&never, 1);
+    tc::fence_barrier_init();
+    s_abort = 0;
+  }
+  __syncthreads();
+  volatile int *abortp = &s_abort;
+  const bool ok = wait_or_abort(&never, 0, abortp, limit);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || s_abort)) {
+    atomicExch(status, kDevTimeout);
+    atomicCAS(status + 1, 0, s_abort - 1);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_bounded_wait_probe(int *status, long long limit_cycles, cudaStream_t st) {
+  bounded_wait_probe_kernel<<<1, 32, 0, st>>>(status, limit_cycles);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches) {
   const SmemMap sm = make_smem_map(p);

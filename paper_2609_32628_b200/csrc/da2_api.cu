@@ -73,6 +73,18 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
 
 bool misaligned(const void *ptr, uintptr_t a) { return ((uintptr_t)ptr % a) != 0; }
 
+// kernels enqueued by the calling thread's last da2_prepare / da2_refresh_operands / da2_attention_fwd
+thread_local int t_last_launches = 0;
+
+// Caller-fixed NVFP4 per-tensor scales travel as kernel arguments (copied when the launch is enqueued, so the call
+// stays legal inside a stream capture; a copy from pageable host memory would not be).
+constexpr int kScaleChunk = 256;
+struct ScaleChunk { float v[kScaleChunk]; };
+__global__ void set_gscale_kernel(float *gscale, int which, int first, int n, ScaleChunk c) {
+  const int i = threadIdx.x;
+  if (i < n) gscale[(size_t)(first + i) * 4 + which] = c.v[i];
+}
+
 }  // namespace
 
 extern "C" {
@@ -81,6 +93,7 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   if (!cfg || !plan_out) return DA2_ERR_INVALID_ARG;
   *plan_out = nullptr;
   if (cfg->B < 1 || cfg->H < 1 || cfg->T < 1 || cfg->Hg < 1 || cfg->Wg < 1) return DA2_ERR_INVALID_ARG;
+  if ((long long)cfg->B * cfg->H > 32767) return DA2_ERR_UNSUPPORTED;  // heads index grid dimensions y and z
   if (cfg->frac16 < 0 || cfg->frac8 < 0 || cfg->frac4 < 0 || cfg->frac16 + cfg->frac8 + cfg->frac4 > 1.0 + 1e-12)
     return DA2_ERR_INVALID_ARG;
   if (!(cfg->lambda >= 0.0f && cfg->lambda <= 1.0f)) return DA2_ERR_INVALID_ARG;
@@ -92,7 +105,6 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   da2_plan_t *plan = new (std::nothrow) da2_plan_t();
   if (!plan) return DA2_ERR_INTERNAL;
   plan->cfg = *cfg;
-  plan->last_launches = 0;
   for (int i = 0; i < 3; ++i) plan->g_host[i] = nullptr;
 
   da2_plan_info_t &I = plan->info;
@@ -190,7 +202,7 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
   da2::Params p = make_params(plan, workspace);
   const da2_plan_info_t &I = plan->info;
   int launches = 0;
-  plan->last_launches = 0;
+  t_last_launches = 0;
   // status word, head maxima and per-channel maxima start at zero (they are contiguous)
   if (cudaMemsetAsync((uint8_t *)workspace + I.off_status, 0, I.off_gscale - I.off_status, st) != cudaSuccess)
     return DA2_ERR_CUDA;
@@ -198,9 +210,14 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
   if (da2::launch_pool(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   for (int i = 0; i < 3; ++i) {  // caller-fixed NVFP4 per-tensor scales replace the derived ones
     if (!plan->g_host[i]) continue;
-    if (cudaMemcpy2DAsync(p.gscale + i, 4 * sizeof(float), plan->g_host[i], sizeof(float), sizeof(float),
-                          (size_t)p.BH, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return DA2_ERR_CUDA;
+    for (int first = 0; first < p.BH; first += kScaleChunk) {
+      ScaleChunk c;
+      const int n = p.BH - first < kScaleChunk ? p.BH - first : kScaleChunk;
+      std::memcpy(c.v, plan->g_host[i] + first, sizeof(float) * (size_t)n);
+      set_gscale_kernel<<<1, kScaleChunk, 0, st>>>(p.gscale, i, first, n, c);
+      if (cudaGetLastError() != cudaSuccess) return DA2_ERR_CUDA;
+      launches += 1;
+    }
   }
   if (select) {
     if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
@@ -209,7 +226,7 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
     if (plan->info.rank_scope != 0 && da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   }
   if (da2::launch_prep(p, qb, kb, vb, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
-  plan->last_launches = launches;
+  t_last_launches = launches;
   return DA2_OK;
 }
 
@@ -233,9 +250,9 @@ da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void
   cudaStream_t st = (cudaStream_t)stream;
   da2::Params p = make_params(plan, const_cast<void *>(workspace));
   int launches = 0;
-  plan->last_launches = 0;
+  t_last_launches = 0;
   if (da2::launch_attention(p, (__nv_bfloat16 *)out, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
-  plan->last_launches = launches;
+  t_last_launches = launches;
   return DA2_OK;
 }
 
@@ -252,7 +269,16 @@ da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, vo
   return DA2_ERR_INTERNAL;
 }
 
-int32_t da2_last_launch_count(const da2_plan_t *plan) { return plan ? plan->last_launches : 0; }
+int32_t da2_last_launch_count(const da2_plan_t *plan) { return plan ? t_last_launches : 0; }
+
+da2_status_t da2_probe_bounded_wait(const da2_plan_t *plan, void *workspace, int64_t limit_cycles, void *stream) {
+  if (!plan || !workspace || limit_cycles < 1 || limit_cycles > 2000000000ll) return DA2_ERR_INVALID_ARG;
+  if (misaligned(workspace, 256)) return DA2_ERR_INVALID_ARG;
+  int *status = (int *)((uint8_t *)workspace + plan->info.off_status);
+  if (da2::launch_bounded_wait_probe(status, (long long)limit_cycles, (cudaStream_t)stream) != cudaSuccess)
+    return DA2_ERR_CUDA;
+  return DA2_OK;
+}
 
 void da2_plan_destroy(da2_plan_t *plan) {
   if (!plan) return;

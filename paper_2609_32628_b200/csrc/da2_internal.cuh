@@ -73,8 +73,9 @@ cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_map_rows(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_order(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
-                        cudaStream_t st, int *launches);
+                        cudaStream_t st, int *launches, bool pool = false);
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);
+cudaError_t launch_bounded_wait_probe(int *status, long long limit_cycles, cudaStream_t st);
 
 }  // namespace da2
 
@@ -82,5 +83,4 @@ struct da2_plan {
   da2_config_t cfg;
   da2_plan_info_t info;
   float *g_host[3];       // optional caller-provided NVFP4 per-tensor scales (copied), or nullptr
-  mutable int last_launches;
 };

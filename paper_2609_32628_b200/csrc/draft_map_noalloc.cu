@@ -53,6 +53,7 @@ extern "C" da2_status_t da2_draft_map_noalloc(const float *q_avg, const float *q
     return DA2_ERR_INVALID_ARG;
   // the fixed scratch array bounds the problem size
   if ((long long)BH * R * R > kMaxLogits || R > 16384) return DA2_ERR_WORKSPACE_TOO_SMALL;
+  if (BH > 32767) return DA2_ERR_UNSUPPORTED;  // heads index grid dimensions y and z of the launches below
   float *scratch = nullptr;
   if (scratch_address(&scratch) != cudaSuccess) return DA2_ERR_CUDA;
 

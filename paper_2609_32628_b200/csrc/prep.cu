@@ -54,7 +54,10 @@ __device__ __forceinline__ uint32_t nvfp4_group(const float (&x)[16], float g, u
   return sc;
 }
 
-template <int D>
+// POOL: the pass also writes the block's average and max descriptors of Q and K (Eq. "v2-descriptors"), so that a
+// call whose quantiser statistics are already known reads Q, K, V from HBM exactly once (Sec. 3.3, "Fused
+// quantization and reordering").
+template <int D, bool POOL>
 __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 *__restrict__ q,
                                                   const __nv_bfloat16 *__restrict__ k,
                                                   const __nv_bfloat16 *__restrict__ v) {
@@ -109,6 +112,28 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
     if (p.tier_active[1]) (tid == 0 ? p.dq8 : p.dk8)[blk] = delta;
   }
   __syncthreads();
+
+  if (POOL) {
+    // one thread per (tensor, channel): sum and maximum over the valid slots of the staged tile.  A sum of at most
+    // 64 bf16 values is exact in fp64, so the mean is correctly rounded whatever the order.
+    const int n_valid = __popcll(mask);
+    for (int idx = tid; idx < 2 * D; idx += NT) {
+      const uint16_t *src = (idx < D ? tq : tk) + (idx % D);
+      double sum = 0.0;
+      float mx = -INFINITY;
+#pragma unroll 8
+      for (int j = 0; j < kSlots; ++j) {
+        if ((mask >> j) & 1ull) {
+          const float x = bf16_to_f32(src[j * D]);
+          sum += (double)x;
+          mx = fmaxf(mx, x);
+        }
+      }
+      const size_t o = blk * D + (idx % D);
+      p.desc[idx < D ? 0 : 2][o] = (float)(sum / (double)n_valid);
+      p.desc[idx < D ? 1 : 3][o] = mx;
+    }
+  }
 
   // ------------------------------------------------------------------ tier 2: BF16, reorder only
   if (p.tier_active[2]) {
@@ -230,21 +255,21 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 }  // namespace
 
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
-                        cudaStream_t st, int *launches) {
+                        cudaStream_t st, int *launches, bool pool) {
   dim3 grid(p.R, p.BH);
   const size_t smem = 3 * (size_t)kSlots * p.d * 2 + 3 * kSfAtomBytes;
+  auto launch = [&](auto kernel) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, NT, smem, st>>>(p, q, k, v);
+    return cudaGetLastError();
+  };
   cudaError_t e;
-  if (p.d == 128) {
-    e = cudaFuncSetAttribute(prep_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    prep_kernel<128><<<grid, NT, smem, st>>>(p, q, k, v);
-  } else {
-    e = cudaFuncSetAttribute(prep_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    prep_kernel<64><<<grid, NT, smem, st>>>(p, q, k, v);
-  }
+  if (p.d == 128) e = pool ? launch(prep_kernel<128, true>) : launch(prep_kernel<128, false>);
+  else e = pool ? launch(prep_kernel<64, true>) : launch(prep_kernel<64, false>);
+  if (e != cudaSuccess) return e;
   *launches += 1;
-  return cudaGetLastError();
+  return cudaSuccess;
 }
 
 }  // namespace da2

@@ -16,10 +16,12 @@ def scale_of(w) -> float:
     return float(np.float32(1.0) / np.sqrt(np.float32(w.head_dim)))
 
 
-def run_gpu(w, q, k, v, rank_scope=0, lam=None, zero_ws=False):
-    """q,k,v CUDA bf16 [B,H,N,d].  Returns (plan, workspace uint8 tensor, out)."""
+def run_gpu(w, q, k, v, rank_scope=0, lam=None, zero_ws=False, g_fixed=None):
+    """q,k,v CUDA bf16 [B,H,N,d].  g_fixed: optional (g_q, g_k, g_v) host arrays [B*H] of caller-fixed NVFP4
+    per-tensor scales.  Returns (plan, workspace uint8 tensor, out)."""
+    gq, gk, gv = (None, None, None) if g_fixed is None else g_fixed
     plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4,
-                        lam=w.lam if lam is None else lam, rank_scope=rank_scope)
+                        lam=w.lam if lam is None else lam, rank_scope=rank_scope, g_q=gq, g_k=gk, g_v=gv)
     ws = (torch.zeros if zero_ws else torch.empty)(int(plan.info.workspace_bytes), dtype=torch.uint8, device=q.device)
     out = torch.full_like(q, float("nan"))
     da2.da2_prepare(plan, q, k, v, ws)
@@ -141,6 +143,21 @@ def oracle_all(w, q, k, v, heads=None, rank_scope=0, lam=None):
                             frac4=w.frac4, head_scope=bool(rank_scope))
     r.update(pl=pl, q=qb, k=kb, v=vb)
     return r
+
+
+def oracle_operands(ref, g_fixed=None, heads=None):
+    """Every quantised operand set of the oracle; with g_fixed = (g_q, g_k, g_v) [BH] the NVFP4 quantisers take those
+    per-tensor scales instead of deriving them (App. C.3: g_X is a given positive per-tensor scale)."""
+    pl = ref["pl"]
+    ops = oracle.quantize_all(ref["q"], ref["k"], ref["v"], pl)
+    if g_fixed is not None:
+        sel = slice(None) if heads is None else list(heads)
+        gq, gk, gv = (np.ascontiguousarray(np.asarray(g, np.float32)[sel]) for g in g_fixed)
+        ops.gq, ops.gk, ops.gv = gq, gk, gv
+        ops.q4, ops.sfq = oracle.quant_nvfp4_qk(ref["q"], pl, gq)
+        ops.k4, ops.sfk = oracle.quant_nvfp4_qk(ref["k"], pl, gk)
+        ops.v4, ops.sfv = oracle.quant_nvfp4_v(ref["v"], pl, gv)
+    return ops
 
 
 def compare_lists(A, ids_o, cnt_o, ids_g, cnt_g, rel=1e-5):

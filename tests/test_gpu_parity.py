@@ -12,7 +12,7 @@ import torch
 import da2_inputs
 import oracle
 import paper_2609_32628_b200 as da2
-from helpers import Workspace, compare_lists, oracle_all, rel_l2, run_gpu, scale_of
+from helpers import Workspace, compare_lists, oracle_all, oracle_operands, rel_l2, run_gpu, scale_of
 
 pytestmark = pytest.mark.gpu
 
@@ -39,7 +39,7 @@ def _inputs(w, device="cuda"):
     return da2_inputs.make_qkv(w, device)
 
 
-def _check_prepare(w, plan, ws, ref, heads=None):
+def _check_prepare(w, plan, ws, ref, heads=None, g_fixed=None):
     V = Workspace(plan, ws, heads)
     I = plan.info
     # descriptors: bit-exact
@@ -67,7 +67,10 @@ def _check_prepare(w, plan, ws, ref, heads=None):
         assert np.array_equal(V.dv8(), dc)
         assert np.array_equal(V.v_e4m3(), codes), "e4m3 v codes"
     if I.tier_active[0]:
-        g = np.stack([oracle.nvfp4_global_scale(ref[n]) for n in ("q", "k", "v")], 1)
+        if g_fixed is None:
+            g = np.stack([oracle.nvfp4_global_scale(ref[n]) for n in ("q", "k", "v")], 1)
+        else:   # caller-fixed per-tensor scales: the workspace must hold exactly those, and the codes follow them
+            g = np.stack([np.asarray(x, np.float32)[V.heads] for x in g_fixed], 1)
         assert np.array_equal(V.gscale(), g)
         for i, which in enumerate(("q", "k")):
             codes, sf = oracle.quant_nvfp4_qk(ref[which], pl, np.ascontiguousarray(g[:, i]))
@@ -87,11 +90,11 @@ def _check_prepare(w, plan, ws, ref, heads=None):
     return bad_rows
 
 
-def _check_attention(w, out, ref, sel, bad_rows, heads=None):
+def _check_attention(w, out, ref, sel, bad_rows, heads=None, g_fixed=None):
     """sel: [(head index within ref, block)]; rows whose lists differ by near-ties are left out."""
     pl = ref["pl"]
     sel = [s for s in sel if tuple(s) not in set(bad_rows)]
-    ops = oracle.quantize_all(ref["q"], ref["k"], ref["v"], pl)
+    ops = oracle_operands(ref, g_fixed, heads)
     exp = oracle.attention(ref["q"], ref["k"], ref["v"], pl, ref["ids"], ref["counts"], ops, scale_of(w), sel)
     dense = oracle.dense(ref["q"], ref["k"], ref["v"], pl, scale_of(w), sel)
     o = out.reshape(-1, w.N, w.head_dim)
@@ -195,46 +198,84 @@ def test_argument_errors_are_reported_before_any_launch():
     assert e.value.code == 1
 
 
-def _sampled_parity(name, nheads=2, nblocks=6):
+def _sampled_parity(name, nheads=2, nblocks=16, rank_scope=0, g_fixed=None):
     """Full-size workload in the launch configuration the benchmark times; the oracle follows on sampled heads
-    (every stage before attention in full for those heads) and on sampled query blocks for the attention output."""
+    (every stage before attention in full for those heads) and on sampled query blocks for the attention output.
+    The sample always holds the first and the last head (the last head's records lie beyond 2^31 bytes in the
+    larger workspaces), both query blocks of two CTA pairs, one block of every edge-tile class and the last block."""
     w = da2_inputs.WORKLOADS[name]
     q, k, v = _inputs(w)
-    plan, ws, out = run_gpu(w, q, k, v)
+    plan, ws, out = run_gpu(w, q, k, v, rank_scope=rank_scope, g_fixed=g_fixed)
     BH, R = w.B * w.H, plan.info.R
     rng = np.random.default_rng(w.seed)
-    heads = sorted(rng.choice(BH, nheads, replace=False).tolist())
-    ref = oracle_all(w, q, k, v, heads=heads)
-    bad = _check_prepare(w, plan, ws, ref, heads=heads)
-    # one block of every edge-tile class plus random ones
+    heads = {0, BH - 1}
+    while len(heads) < min(nheads, BH):
+        heads.add(int(rng.integers(BH)))
+    heads = sorted(heads)[:max(nheads, 1)] if nheads < 2 else sorted(heads)
+    ref = oracle_all(w, q, k, v, heads=heads, rank_scope=rank_scope)
+    bad = _check_prepare(w, plan, ws, ref, heads=heads, g_fixed=g_fixed)
     R_f, ntx = plan.info.R_f, plan.info.ntx
-    blocks = {0, ntx - 1, R_f - ntx, R_f - 1, R - 1} | set(rng.choice(R, nblocks, replace=False).tolist())
+    pair0, pair1 = 2 * int(rng.integers(R // 2)), 2 * int(rng.integers(R // 2))
+    blocks = {0, ntx - 1, R_f - ntx, R_f - 1, R - 1, pair0, pair0 + 1, pair1, pair1 + 1}
+    while len(blocks) < min(nblocks, R):
+        blocks.add(int(rng.integers(R)))
     sel = [(hi, int(a)) for hi in range(len(heads)) for a in sorted(blocks)]
-    _check_attention(w, out, ref, sel, bad, heads=heads)
+    _check_attention(w, out, ref, sel, bad, heads=heads, g_fixed=g_fixed)
 
 
 def test_wan1p3b_480p_sampled_parity():
-    _sampled_parity("wan1p3b_480p", nheads=2, nblocks=6)
+    _sampled_parity("wan1p3b_480p", nheads=3, nblocks=16)
+
+
+def test_wan1p3b_480p_head_scope_sampled_parity():
+    """Alg. 1 as printed (one ranking over all R*R pairs of a head) at a full-size configuration: rows of very
+    different lengths, the scheduling order, CSR-style list offsets."""
+    _sampled_parity("wan1p3b_480p", nheads=2, nblocks=16, rank_scope=1)
 
 
 def test_hunyuan_720p_sampled_parity():
-    _sampled_parity("hunyuan_720p", nheads=1, nblocks=4)
+    _sampled_parity("hunyuan_720p", nheads=2, nblocks=16)
 
 
 def test_wan14b_720p_sampled_parity():
     """The benchmark's workload (20 % 8-bit + 40 % 4-bit, K outlier channels) in the benchmark's launch configuration."""
-    _sampled_parity("wan14b_720p", nheads=1, nblocks=4)
+    _sampled_parity("wan14b_720p", nheads=2, nblocks=16)
 
 
 def test_wan14b_720p_bf16_8bit_variant_sampled_parity():
-    _sampled_parity("wan14b_720p_hi", nheads=1, nblocks=4)
+    _sampled_parity("wan14b_720p_hi", nheads=2, nblocks=16)
 
 
-def test_sweep_point_sampled_parity():
-    """One point of the budget sweep: 16 x 48 x 48 grid, 24 heads, 10 % 8-bit + 40 % 4-bit."""
-    w = da2_inputs.sweep_workload(2, 0.10, 0.40)
+@pytest.mark.parametrize("grid,high,low", [(2, 0.10, 0.40), (1, 0.0, 0.40), (3, 0.20, 0.0), (0, 0.05, 0.60)])
+def test_sweep_point_sampled_parity(grid, high, low):
+    """Points of the budget sweep (24 heads, d = 128): a mixed point, a point without the 8-bit tier, a point
+    without the 4-bit tier, and the smallest grid at the largest 4-bit share."""
+    w = da2_inputs.sweep_workload(grid, high, low)
     da2_inputs.WORKLOADS[w.name] = w
-    _sampled_parity(w.name, nheads=1, nblocks=4)
+    _sampled_parity(w.name, nheads=2, nblocks=12)
+
+
+@pytest.mark.parametrize("name", ["sweep_131k_all8", "sweep_131k_allbf16"])
+def test_sweep_dense_endpoints_sampled_parity(name):
+    """The two zero-sparsity endpoints of the sweep at the largest grid (131,072 tokens): every key block retained in
+    the 8-bit tier, and every key block retained in bf16 (which the oracle's pins tie to dense attention)."""
+    _sampled_parity(name, nheads=2, nblocks=8)
+
+
+def test_caller_fixed_nvfp4_scales():
+    """g_q, g_k, g_v supplied by the caller (App. C.3: a given positive per-tensor scale): the workspace holds exactly
+    those scales, codes and group scales are the oracle's for the same g, and so is the attention output.  One of
+    the scales is deliberately too small, so that the largest groups saturate at the top scale code."""
+    w = SMALL["ragged3"]
+    BH = w.B * w.H
+    g_fixed = ([0.004, 0.0035], [0.0011, 0.005], [0.003, 0.0042])
+    assert all(len(g) == BH for g in g_fixed)
+    q, k, v = _inputs(w)
+    plan, ws, out = run_gpu(w, q, k, v, g_fixed=g_fixed)
+    ref = oracle_all(w, q, k, v)
+    bad = _check_prepare(w, plan, ws, ref, g_fixed=g_fixed)
+    sel = [(h, a) for h in range(BH) for a in range(plan.info.R)]
+    _check_attention(w, out, ref, sel, bad, g_fixed=g_fixed)
 
 
 def test_refresh_operands_keeps_the_selection():
@@ -292,6 +333,26 @@ def test_prepare_and_attention_replay_from_a_cuda_graph():
         torch.cuda.synchronize()
         assert da2.da2_device_status(plan, ws2) == 0
         assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+
+
+def test_graph_replay_with_caller_fixed_scales():
+    """With caller-fixed NVFP4 scales da2_prepare hands them over as kernel arguments (no copy from pageable host
+    memory), so the call can still be captured; the replay gives the bits of the eager call."""
+    w = SMALL["ragged3"]
+    g_fixed = ([0.004, 0.0035], [0.0011, 0.005], [0.003, 0.0042])
+    q, k, v = _inputs(w)
+    plan, ws, out = run_gpu(w, q, k, v, zero_ws=True, g_fixed=g_fixed)
+    ws2 = torch.zeros_like(ws)
+    out2 = torch.full_like(out, float("nan"))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        da2.da2_prepare(plan, q, k, v, ws2)
+        da2.da2_attention_fwd(plan, q, k, v, ws2, out2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert da2.da2_device_status(plan, ws2) == 0
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    assert torch.equal(ws2, ws)
 
 
 def test_host_pipeline_equals_the_direct_call():

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import da2_inputs
+import oracle
 import paper_2609_32628_b200 as da2
 
 pytestmark = pytest.mark.gpu
@@ -40,8 +41,11 @@ def test_noalloc_draft_map_matches_regular_path_twice_in_a_row():
     torch.cuda.synchronize()
     for out, (desc, ref, lam, scale) in zip(outs, prepared):
         assert torch.isfinite(out).all()
-        assert np.allclose(out.cpu().numpy(), ref.cpu().numpy(), rtol=2e-5, atol=1e-12)
+        assert torch.equal(out, ref)   # the same kernels on the same descriptors: identical bits
         assert np.allclose(out.sum(-1).cpu().numpy(), 1.0, atol=1e-5)
+        # and against the CPU oracle's draft map of the same descriptors (the tolerance of the regular parity tests)
+        exp = oracle.draft(*(t.cpu().numpy() for t in desc), lam, scale)
+        assert np.allclose(out.cpu().numpy(), exp, rtol=2e-5, atol=1e-12)
 
 
 def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
@@ -57,3 +61,5 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
                    vp, vp]
     rc = fn(*(int(t.data_ptr()) for t in desc), BH, R, d, 0.2, 0.125, int(x.data_ptr()), None)
     assert rc == 3  # DA2_ERR_WORKSPACE_TOO_SMALL, nothing launched
+    rc = fn(*(int(t.data_ptr()) for t in desc), 40000, 5, d, 0.2, 0.125, int(x.data_ptr()), None)
+    assert rc == 2  # DA2_ERR_UNSUPPORTED: more heads than a launch dimension holds, nothing launched
