@@ -187,6 +187,16 @@ def quant_v_e4m3(v: np.ndarray, pl: Plan):
     return codes, delta_c
 
 
+def quant_v_e4m3_given(v: np.ndarray, pl: Plan, delta_c: np.ndarray) -> np.ndarray:
+    """E4M3 codes of V under a given per-(head, channel) scale delta_c [BH, d] (0 = channel skipped)."""
+    BH, N, d = v.shape
+    codes = np.empty((BH, pl.R, pl.S, d), np.uint8)
+    dc = np.ascontiguousarray(delta_c, np.float32)
+    lib().orc_quant_v_e4m3_given(_p(v), _i64(BH), _i64(N), _i(d), _i(pl.R), _i(pl.S), _p(pl.slot_token), _p(dc),
+                                 _p(codes))
+    return codes
+
+
 def nvfp4_global_scale(x: np.ndarray) -> np.ndarray:
     BH, N, d = x.shape
     g = np.empty((BH,), np.float32)

@@ -316,6 +316,29 @@ void orc_quant_v_e4m3(const uint16_t *v, i64 BH, i64 N, int d, int R, int S, con
   }
 }
 
+/* E4M3 values of the 8-bit path with a GIVEN per-(head, channel) scale delta_c (App. C.3 takes
+ * delta_c = max_v |V_vc| / 2.25 from the tensor itself; a caller may instead carry the scale of an
+ * earlier, similar tensor over, e.g. of the previous denoising step: the cast is the same, only the
+ * scale's origin differs).  code = cast_E4M3(fl32(V / delta_c)); delta_c = 0 marks a skipped channel. */
+void orc_quant_v_e4m3_given(const uint16_t *v, i64 BH, i64 N, int d, int R, int S, const int32_t *slot_token,
+                            const float *delta_c, uint8_t *codes) {
+#pragma omp parallel for schedule(static)
+  for (i64 bh = 0; bh < BH; ++bh)
+    for (int a = 0; a < R; ++a)
+      for (int j = 0; j < S; ++j) {
+        int tok = slot_token[(i64)a * S + j];
+        for (int c = 0; c < d; ++c) {
+          uint8_t code = 0;
+          float dl = delta_c[bh * d + c];
+          if (tok >= 0 && dl > 0.0f) {
+            volatile float r = bf16_bits_to_f32(v[(bh * N + tok) * d + c]) / dl;
+            code = orc_cast_e4m3(r);
+          }
+          codes[((bh * R + a) * S + j) * d + c] = code;
+        }
+      }
+}
+
 /* per-head max |x| over all valid tokens, and the derived NVFP4 per-tensor scale
  * g = amax / 2688 (so the largest group scale encodes as 448); g = 1 for a zero head. */
 void orc_nvfp4_global_scale(const uint16_t *x, i64 BH, i64 N, int d, float *g) {

@@ -322,6 +322,32 @@ def test_v_e4m3_quantiser():
     assert oracle.decode_e4m3(amax_code) == 2.25
 
 
+def test_v_e4m3_quantiser_with_a_given_scale():
+    """The given-scale variant: (i) fed the tensor's own max/2.25 it returns the codes of the self-scaled quantiser,
+    (ii) under any other scale every code is torch's float8_e4m3fn cast of fl32(V / delta) (saturating at 448, which
+    a too small scale reaches), (iii) a zero scale skips the channel."""
+    rng = np.random.default_rng(29)
+    pl = oracle.plan(2, 12, 20)
+    v = rand_bf16(rng, (2, pl.N, 16), 3.0)
+    codes_self, dc = oracle.quant_v_e4m3(bits(v), pl)
+    assert np.array_equal(oracle.quant_v_e4m3_given(bits(v), pl, dc), codes_self)
+    other = (dc * rng.uniform(0.002, 3.0, dc.shape)).astype(np.float32)
+    other[1, 5] = 0.0
+    other[0, 3] = dc[0, 3] * np.float32(0.001)   # far too small: the larger values of this channel saturate
+    codes = oracle.quant_v_e4m3_given(bits(v), pl, other)
+    vf = v.float().numpy()
+    st = np.maximum(pl.slot_token, 0)
+    valid = (pl.slot_token >= 0)[None, :, :, None]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ratio = (vf[:, st] / other[:, None, None, :]).astype(np.float32)
+    ratio = np.clip(np.nan_to_num(ratio, nan=0.0, posinf=448.0, neginf=-448.0), -448.0, 448.0)
+    ref = torch.from_numpy(ratio).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    live = valid & (other > 0)[:, None, None, :]
+    assert np.array_equal(np.where(live, codes, 0), np.where(live, ref, 0))
+    assert (codes[~np.broadcast_to(live, codes.shape)] == 0).all()
+    assert (np.abs(ratio[np.broadcast_to(live, ratio.shape)]) >= 448.0).any()   # the saturating branch is exercised
+
+
 def test_nvfp4_quantisers():
     rng = np.random.default_rng(10)
     pl = oracle.plan(1, 16, 12)
