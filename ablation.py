@@ -2,11 +2,11 @@
 precision budgets and draft-map mixing weights (the shape of the paper's budget / lambda studies, Sec. 4 and Fig. 5,
 without its models or datasets).
 
-    python -m paper_2609_32628_b200.ablation [--grid T,Hg,Wg] [--heads H] [--blocks 8] [--steps 3]
+    python ablation.py [--grid T,Hg,Wg] [--heads H] [--blocks 8] [--steps 3]
 
-Every line is one configuration run through da2_prepare + da2_attention_fwd on cuda:0.  The error is the relative L2
-distance to dense softmax attention (fp32 matmuls in PyTorch, evaluated for a sample of query blocks of every head:
-that reference is the plain definition and only serves this report).  Prints a markdown table.
+A report script beside bench.py, not part of the library.  Every line is one configuration run through da2_prepare +
+da2_attention_fwd on cuda:0.  The error is the relative L2 distance to dense softmax attention written out as its
+definition with fp64 PyTorch matmuls, for a sample of query blocks of every head.  Prints a markdown table.
 """
 from __future__ import annotations
 
@@ -17,7 +17,7 @@ import sys
 
 import torch
 
-sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 import da2_inputs  # noqa: E402
 from paper_2609_32628_b200 import binding as da2  # noqa: E402
 
@@ -31,11 +31,12 @@ LAMBDAS = (0.0, 0.2, 0.5, 1.0)  # weight of the max-pooled branch in the draft m
 
 
 def dense_rows(q, k, v, rows, scale):
-    """softmax(q_rows k^T * scale) v for token index tensor `rows` [n] of every head; fp32."""
-    qs = q[0, :, rows].float()                                    # [H, n, d]
-    s = torch.einsum("hnd,hmd->hnm", qs, k[0].float()) * scale
-    p = torch.softmax(s, dim=-1)
-    return torch.einsum("hnm,hmd->hnd", p, v[0].float())
+    """softmax(q_rows k^T * scale) v for token index tensor `rows` [n] of every head; fp64, head by head."""
+    out = []
+    for h in range(q.shape[1]):
+        s = (q[0, h, rows].double() @ k[0, h].double().t()) * scale
+        out.append(torch.softmax(s, dim=-1) @ v[0, h].double())
+    return torch.stack(out).float()
 
 
 def block_tokens(w, blocks):

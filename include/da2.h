@@ -135,6 +135,21 @@ da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, c
 da2_status_t da2_refresh_operands(const da2_plan_t *plan, const void *q, const void *k, const void *v,
                                   void *workspace, size_t workspace_bytes, void *stream);
 
+/* Single-pass preparation under known quantiser statistics (Sec. 3.3, "Fused quantization and reordering": spatial
+ * gathering, average- and max-pooling and quantisation fused so that the token features cross global memory once).
+ * da2_prepare needs two passes over Q, K, V, because the NVFP4 per-tensor scales g_X and the E4M3 per-channel value
+ * scales delta_c^V (App. C.3) are statistics of the whole head that must exist before any block is quantised.  This
+ * call does not derive them: it quantises with the scales that are in the workspace -- left there by an earlier
+ * da2_prepare / da2_refresh_operands with this plan, typically for the previous denoising step or layer, whose
+ * activations have nearly the same range -- and writes region descriptors and every operand record in ONE pass
+ * (INT8 block scales are local to a block and are always derived).  A value beyond the carried-over range saturates
+ * in its format exactly as the casts define.  reselect != 0: the draft map, the ranking and the lists are then
+ * recomputed from the new descriptors; reselect == 0: the earlier selection is kept (as da2_refresh_operands does).
+ * The scales and statistics in the workspace are left untouched, so da2_attention_fwd dequantises with the scales
+ * the records were made with.  Same argument rules as da2_prepare.  Enqueues on stream. */
+da2_status_t da2_prepare_cached_scales(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                                       void *workspace, size_t workspace_bytes, int32_t reselect, void *stream);
+
 /* Phased mixed-precision block-sparse attention.  workspace must have been filled by da2_prepare for the same
  * q, k, v (ordering on the same stream is enough).  Rows whose list is empty give zeros (App. C.1). */
 da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,

@@ -64,6 +64,8 @@ def load_library():
         lib.da2_prepare.argtypes = [vp, vp, vp, vp, vp, sz, vp]
         lib.da2_refresh_operands.restype = ctypes.c_int
         lib.da2_refresh_operands.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+        lib.da2_prepare_cached_scales.restype = ctypes.c_int
+        lib.da2_prepare_cached_scales.argtypes = [vp, vp, vp, vp, vp, sz, ctypes.c_int32, vp]
         lib.da2_attention_fwd.restype = ctypes.c_int
         lib.da2_attention_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         lib.da2_device_status.restype = ctypes.c_int
@@ -154,6 +156,15 @@ def da2_refresh_operands(plan: Plan, q, k, v, workspace, stream=None) -> None:
                                     workspace.numel() * workspace.element_size(), _stream(stream))
     if rc != 0:
         raise Da2Error(rc, "da2_refresh_operands")
+
+
+def da2_prepare_cached_scales(plan: Plan, q, k, v, workspace, reselect: bool = True, stream=None) -> None:
+    """Single-pass preparation with the NVFP4 per-tensor and E4M3 per-channel scales already in the workspace."""
+    rc = load_library().da2_prepare_cached_scales(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(workspace),
+                                                  workspace.numel() * workspace.element_size(),
+                                                  1 if reselect else 0, _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_prepare_cached_scales")
 
 
 def da2_attention_fwd(plan: Plan, q, k, v, workspace, out, stream=None) -> None:

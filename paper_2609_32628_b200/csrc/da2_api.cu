@@ -242,6 +242,30 @@ da2_status_t da2_refresh_operands(const da2_plan_t *plan, const void *q, const v
   return prepare_impl(plan, q, k, v, workspace, workspace_bytes, stream, false);
 }
 
+da2_status_t da2_prepare_cached_scales(const da2_plan_t *plan, const void *q, const void *k, const void *v,
+                                       void *workspace, size_t workspace_bytes, int32_t reselect, void *stream) {
+  if (!plan || !q || !k || !v || !workspace) return DA2_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(workspace, 256))
+    return DA2_ERR_INVALID_ARG;
+  if (workspace_bytes < plan->info.workspace_bytes) return DA2_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  da2::Params p = make_params(plan, workspace);
+  int launches = 0;
+  t_last_launches = 0;
+  // only the status word is cleared: the statistics and the scales derived from them stay as the earlier call left them
+  if (cudaMemsetAsync((uint8_t *)workspace + plan->info.off_status, 0, 64 * sizeof(int), st) != cudaSuccess)
+    return DA2_ERR_CUDA;
+  const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k, *vb = (const __nv_bfloat16 *)v;
+  if (da2::launch_prep(p, qb, kb, vb, st, &launches, /*pool=*/true) != cudaSuccess) return DA2_ERR_CUDA;
+  if (reselect) {
+    if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (plan->info.rank_scope != 0 && da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+  }
+  t_last_launches = launches;
+  return DA2_OK;
+}
+
 da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,
                                const void *workspace, void *out, void *stream) {
   if (!plan || !q || !k || !v || !workspace || !out) return DA2_ERR_INVALID_ARG;

@@ -145,7 +145,7 @@ def oracle_all(w, q, k, v, heads=None, rank_scope=0, lam=None):
     return r
 
 
-def oracle_operands(ref, g_fixed=None, heads=None):
+def oracle_operands(ref, g_fixed=None, heads=None, dv_fixed=None):
     """Every quantised operand set of the oracle; with g_fixed = (g_q, g_k, g_v) [BH] the NVFP4 quantisers take those
     per-tensor scales instead of deriving them (App. C.3: g_X is a given positive per-tensor scale)."""
     pl = ref["pl"]
@@ -157,6 +157,10 @@ def oracle_operands(ref, g_fixed=None, heads=None):
         ops.q4, ops.sfq = oracle.quant_nvfp4_qk(ref["q"], pl, gq)
         ops.k4, ops.sfk = oracle.quant_nvfp4_qk(ref["k"], pl, gk)
         ops.v4, ops.sfv = oracle.quant_nvfp4_v(ref["v"], pl, gv)
+    if dv_fixed is not None:   # carried-over E4M3 per-channel value scales [BH, d]
+        sel = slice(None) if heads is None else list(heads)
+        ops.dv8 = np.ascontiguousarray(np.asarray(dv_fixed, np.float32)[sel])
+        ops.v8 = oracle.quant_v_e4m3_given(ref["v"], pl, ops.dv8)
     return ops
 
 

@@ -39,7 +39,7 @@ def _inputs(w, device="cuda"):
     return da2_inputs.make_qkv(w, device)
 
 
-def _check_prepare(w, plan, ws, ref, heads=None, g_fixed=None):
+def _check_prepare(w, plan, ws, ref, heads=None, g_fixed=None, dv_fixed=None):
     V = Workspace(plan, ws, heads)
     I = plan.info
     # descriptors: bit-exact
@@ -63,7 +63,11 @@ def _check_prepare(w, plan, ws, ref, heads=None, g_fixed=None):
             codes, delta = oracle.quant_int8(x, pl)
             assert np.array_equal(V.q_or_k_int8(which), codes), f"int8 {which} codes"
             assert np.array_equal(V.dq8() if which == "q" else V.dk8(), delta), f"int8 {which} scales"
-        codes, dc = oracle.quant_v_e4m3(ref["v"], pl)
+        if dv_fixed is None:
+            codes, dc = oracle.quant_v_e4m3(ref["v"], pl)
+        else:   # carried-over per-channel scales: the workspace still holds them, the codes follow them
+            dc = np.ascontiguousarray(np.asarray(dv_fixed, np.float32)[V.heads])
+            codes = oracle.quant_v_e4m3_given(ref["v"], pl, dc)
         assert np.array_equal(V.dv8(), dc)
         assert np.array_equal(V.v_e4m3(), codes), "e4m3 v codes"
     if I.tier_active[0]:
@@ -90,11 +94,11 @@ def _check_prepare(w, plan, ws, ref, heads=None, g_fixed=None):
     return bad_rows
 
 
-def _check_attention(w, out, ref, sel, bad_rows, heads=None, g_fixed=None):
+def _check_attention(w, out, ref, sel, bad_rows, heads=None, g_fixed=None, dv_fixed=None):
     """sel: [(head index within ref, block)]; rows whose lists differ by near-ties are left out."""
     pl = ref["pl"]
     sel = [s for s in sel if tuple(s) not in set(bad_rows)]
-    ops = oracle_operands(ref, g_fixed, heads)
+    ops = oracle_operands(ref, g_fixed, heads, dv_fixed)
     exp = oracle.attention(ref["q"], ref["k"], ref["v"], pl, ref["ids"], ref["counts"], ops, scale_of(w), sel)
     dense = oracle.dense(ref["q"], ref["k"], ref["v"], pl, scale_of(w), sel)
     o = out.reshape(-1, w.N, w.head_dim)
@@ -305,6 +309,44 @@ def test_refresh_operands_keeps_the_selection():
     assert _check_prepare(w2, plan, ws, mixed) == bad
     sel = [(h, a) for h in range(w1.B * w1.H) for a in range(I.R)]
     _check_attention(w2, out, mixed, sel, bad)
+    assert torch.isfinite(out.float()).all()
+
+
+@pytest.mark.parametrize("reselect", [True, False])
+def test_prepare_cached_scales_is_one_pass_with_carried_over_scales(reselect):
+    """da2_prepare_cached_scales: descriptors and every operand record of NEW inputs in one pass, quantised with the
+    NVFP4 per-tensor and E4M3 per-channel scales an earlier da2_prepare left in the workspace (Sec. 3.3, fused
+    gathering + pooling + quantisation).  The new Q and K (and four channels of V) are 1.6 times larger, so values
+    beyond the carried-over range occur and must saturate as the casts define.  Everything is compared with the oracle fed the same
+    scales; the scales in the workspace must not change."""
+    w1 = SMALL["ragged3"]
+    w2 = W("ragged3b", w1.B, w1.H, w1.head_dim, w1.T, w1.Hg, w1.Wg, w1.frac16, w1.frac8, w1.frac4, seed=211)
+    q1, k1, v1 = _inputs(w1)
+    q2, k2, v2 = _inputs(w2)
+    q2, k2 = ((x.float() * 1.6).to(torch.bfloat16) for x in (q2, k2))
+    gain = torch.ones(w1.head_dim, device="cuda")
+    gain[[5, 40, 77, 100]] = 1.6          # a few value channels leave the carried-over range as well
+    v2 = (v2.float() * gain).to(torch.bfloat16)
+    plan, ws, _ = run_gpu(w1, q1, k1, v1, zero_ws=True)
+    ref1 = oracle_all(w1, q1, k1, v1)
+    bad1 = _check_prepare(w1, plan, ws, ref1)
+    V1 = Workspace(plan, ws)
+    g1, dv1 = V1.gscale().copy(), V1.dv8().copy()
+    g_fixed = (g1[:, 0], g1[:, 1], g1[:, 2])
+    out = torch.full_like(q2, float("nan"))
+    da2.da2_prepare_cached_scales(plan, q2, k2, v2, ws, reselect=reselect)
+    assert da2.da2_last_launch_count(plan) == (3 if reselect else 1)   # one pass over Q, K, V (+ draft map, ranking)
+    da2.da2_attention_fwd(plan, q2, k2, v2, ws, out)
+    torch.cuda.synchronize()
+    assert da2.da2_device_status(plan, ws) == 0
+    ref2 = oracle_all(w2, q2, k2, v2)
+    if not reselect:   # the earlier call's selection stays
+        ref2.update(A=ref1["A"], ids=ref1["ids"], counts=ref1["counts"], tags=ref1["tags"])
+    bad = _check_prepare(w2, plan, ws, ref2, g_fixed=g_fixed, dv_fixed=dv1)
+    if not reselect:
+        assert bad == bad1
+    sel = [(h, a) for h in range(w1.B * w1.H) for a in range(plan.info.R)]
+    _check_attention(w2, out, ref2, sel, bad, g_fixed=g_fixed, dv_fixed=dv1)
     assert torch.isfinite(out.float()).all()
 
 
