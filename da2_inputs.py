@@ -144,6 +144,10 @@ def _register_sweep():
             w = sweep_workload(gi, high, low)
             WORKLOADS[f"sweep_{names[gi]}_{int(high * 100)}_{int(low * 100)}"] = Workload(
                 **{**w.__dict__, "name": f"sweep_{names[gi]}_{int(high * 100)}_{int(low * 100)}"})
+    # single-tier calls at the middle grid (every block kept in one format): small enough for a profiler capture
+    for name, w in (("sweep_37k_all4", sweep_workload(2, 0.0, 1.0)), ("sweep_37k_all8", sweep_workload(2, 1.0, 0.0)),
+                    ("sweep_37k_allbf16", sweep_workload(2, 1.0, 0.0, high_is_bf16=True))):
+        WORKLOADS[name] = Workload(**{**w.__dict__, "name": name})
     w = sweep_workload(4, 1.0, 0.0)
     WORKLOADS["sweep_131k_all8"] = Workload(**{**w.__dict__, "name": "sweep_131k_all8"})
     w = sweep_workload(4, 1.0, 0.0, high_is_bf16=True)

@@ -107,10 +107,12 @@ class Plan:
     S: int
     slot_token: np.ndarray  # int32 [R, S], -1 = padding
     n_valid: np.ndarray     # int32 [R]
+    n_prefix: int = 0       # prefix (text) tokens in front of the video tokens; their blocks follow the video regions
+    R_video: int = -1       # number of video regions (== R without a prefix)
 
     @property
     def N(self) -> int:
-        return self.T * self.Hg * self.Wg
+        return self.T * self.Hg * self.Wg + self.n_prefix
 
 
 def plan(T: int, Hg: int, Wg: int, th: int = 8, tw: int = 8) -> Plan:
@@ -120,6 +122,61 @@ def plan(T: int, Hg: int, Wg: int, th: int = 8, tw: int = 8) -> Plan:
     nv = np.empty((R,), np.int32)
     lib().orc_plan(_i(T), _i(Hg), _i(Wg), _i(th), _i(tw), _p(st), _p(nv))
     return Plan(T, Hg, Wg, th, tw, R, S, st, nv)
+
+
+# ---------------------------------------------------------------- prefix tokens
+# App. C.1: "prefix interactions lie outside the video-region budget": a video query keeps every valid prefix key,
+# a prefix query attends to everything.  Readings: the P prefix tokens come first in the token order, followed by the
+# video tokens in raster order; prefix tokens form ceil(P/S) blocks of S consecutive tokens that follow the video
+# regions in the block numbering; prefix interactions run in the 16-bit tier (they are "retained prefix
+# interactions" of a precision set, Sec. 3.2, and no lower format is named for them), i.e. last in the phase order.
+def plan_with_prefix(pl: Plan, P: int) -> Plan:
+    """Block table of the joint sequence [P prefix tokens | video tokens]: video regions (token ids shifted by P),
+    then the prefix blocks."""
+    assert pl.n_prefix == 0
+    if P == 0:
+        return Plan(pl.T, pl.Hg, pl.Wg, pl.th, pl.tw, pl.R, pl.S, pl.slot_token, pl.n_valid, 0, pl.R)
+    Rp = -(-P // pl.S)
+    st = np.full((pl.R + Rp, pl.S), -1, np.int32)
+    st[:pl.R] = np.where(pl.slot_token >= 0, pl.slot_token + P, -1)
+    for j in range(Rp):
+        toks = np.arange(j * pl.S, min(P, (j + 1) * pl.S), dtype=np.int32)
+        st[pl.R + j, :len(toks)] = toks
+    nv = (st >= 0).sum(1).astype(np.int32)
+    return Plan(pl.T, pl.Hg, pl.Wg, pl.th, pl.tw, pl.R + Rp, pl.S, st, nv, P, pl.R)
+
+
+def lists_with_prefix(ids: np.ndarray, counts: np.ndarray, R: int, Rp: int):
+    """Lists of the joint sequence from the ranked video lists ids [BH,R,*], counts [BH,R,3]: every video row gets
+    all prefix blocks appended to its 16-bit segment, every prefix row keeps all blocks in the 16-bit tier."""
+    BH = ids.shape[0]
+    Rt = R + Rp
+    out = np.full((BH, Rt, Rt), -1, np.int32)
+    cnt = np.zeros((BH, Rt, 3), np.int32)
+    pre = np.arange(R, Rt, dtype=np.int32)
+    for h in range(BH):
+        for a in range(R):
+            n = int(counts[h, a].sum())
+            out[h, a, :n] = ids[h, a, :n]
+            out[h, a, n:n + Rp] = pre
+            cnt[h, a] = counts[h, a] + np.array([0, 0, Rp], np.int32)
+        for a in range(R, Rt):
+            out[h, a] = np.arange(Rt, dtype=np.int32)
+            cnt[h, a] = (0, 0, Rt)
+    return out, cnt
+
+
+def pad_operands(ops: "Operands", Rt: int) -> "Operands":
+    """Per-block operand arrays padded with empty entries for the prefix blocks (which only ever run in the 16-bit
+    tier and therefore have no quantised operands)."""
+    def pad(x):
+        if x.ndim < 2 or x.shape[1] == Rt:
+            return x
+        shape = list(x.shape)
+        shape[1] = Rt - x.shape[1]
+        return np.ascontiguousarray(np.concatenate([x, np.zeros(shape, x.dtype)], 1))
+    keep = {"dv8", "gq", "gk", "gv"}   # per head (and channel), not per block
+    return Operands(**{k: (v if k in keep else pad(v)) for k, v in ops.__dict__.items()})
 
 
 def quotas(f16: float, f8: float, f4: float, M: int):

@@ -686,6 +686,94 @@ def test_online_nvfp4_weight_quantiser_is_the_printed_formula(grid, mix):
     assert n_checked > 200 and n_nonuniform > 10
 
 
+def _prefix_case(rng, P, mix, d=32, grid=(2, 12, 20)):
+    """Joint tensors [P prefix | video], the video-only stages on the video part, lists and plan of the joint
+    sequence."""
+    plv = oracle.plan(*grid)
+    q, k, v = (rand_bf16(rng, (1, P + plv.N, d), 1.5), rand_bf16(rng, (1, P + plv.N, d)),
+               rand_bf16(rng, (1, P + plv.N, d)))
+    vid = lambda t: np.ascontiguousarray(bits(t)[:, P:])
+    ops = oracle.quantize_all(vid(q), vid(k), vid(v), plv)
+    ids, counts = _mixed_lists(rng, 1, plv.R, *mix)
+    pl = oracle.plan_with_prefix(plv, P)
+    ids_x, cnt_x = oracle.lists_with_prefix(ids, counts, plv.R, pl.R - plv.R)
+    return plv, pl, q, k, v, oracle.pad_operands(ops, pl.R), ids, counts, ids_x, cnt_x
+
+
+def test_prefix_plan_is_a_partition_of_the_joint_sequence():
+    plv = oracle.plan(2, 12, 20)
+    for P in (0, 1, 64, 77, 200):
+        pl = oracle.plan_with_prefix(plv, P)
+        toks = pl.slot_token[pl.slot_token >= 0]
+        assert np.array_equal(np.sort(toks), np.arange(P + plv.N))
+        assert pl.R == plv.R + -(-P // 64) and pl.N == P + plv.N
+        assert np.array_equal(pl.slot_token[:plv.R][plv.slot_token >= 0], plv.slot_token[plv.slot_token >= 0] + P)
+        if P:
+            assert np.array_equal(pl.slot_token[plv.R:].reshape(-1)[:P], np.arange(P))
+
+
+def test_prefix_keys_alone_and_prefix_queries_dense():
+    """App. C.1.  (i) With every video block skipped, a video query attends to the prefix keys alone: its output is
+    dense softmax attention over those P keys (fp64, written out here).  (ii) A prefix query is non-sparse: its row
+    equals dense attention over the whole joint sequence.  Only the bf16 rounding of the weights (16-bit tier) and of
+    the output separates the two sides."""
+    rng = np.random.default_rng(31)
+    P, d = 77, 32
+    plv, pl, q, k, v, ops, ids, counts, ids_x, cnt_x = _prefix_case(rng, P, (0, 0, 0), d)
+    s = 1 / math.sqrt(d)
+    Q, K, V = f64(q)[0], f64(k)[0], f64(v)[0]
+    sel = [(0, 0), (0, 5), (0, plv.R - 1)]
+    out = oracle.attention(bits(q), bits(k), bits(v), pl, ids_x, cnt_x, ops, s, sel)
+    for i, (_, a) in enumerate(sel):
+        for j in range(64):
+            u = pl.slot_token[a, j]
+            if u < 0:
+                assert (out[i, j] == 0).all()
+                continue
+            lg = K[:P] @ Q[u] * s
+            w = np.exp(lg - lg.max())
+            ref = (w / w.sum()) @ V[:P]
+            assert np.abs(out[i, j] - ref).max() <= 2.0 ** -7 * max(1.0, np.abs(ref).max())
+    pre_rows = [(0, a) for a in range(plv.R, pl.R)]
+    got = oracle.attention(bits(q), bits(k), bits(v), pl, ids_x, cnt_x, ops, s, pre_rows)
+    dense = oracle.dense(bits(q), bits(k), bits(v), pl, s, pre_rows)
+    assert np.abs(got - dense).max() <= 2.0 ** -7 * max(1.0, np.abs(dense).max())
+    assert (got[-1, P - 64:] == 0).all()          # slots of the last prefix block beyond token P-1 are padding
+
+
+def test_prefix_blocks_sit_outside_the_budget_and_vanish_without_prefix():
+    """(i) P = 0 leaves the joint tables identical to the video ones and the output bit-identical.  (ii) With a
+    prefix, every video row keeps exactly its ranked blocks plus all prefix blocks, the latter in the 16-bit segment
+    (last in the phase order), so the budget counts of the quantised tiers do not change.  (iii) The output equals
+    the per-key reconstruction sum(what * vhat) / ell over the retained video keys AND the P prefix keys."""
+    rng = np.random.default_rng(32)
+    d = 32
+    plv, pl0, q, k, v, ops0, ids, counts, ids0, cnt0 = _prefix_case(rng, 0, (3, 2, 1), d)
+    s = 1 / math.sqrt(d)
+    sel = [(0, 1), (0, 4)]
+    base = oracle.attention(bits(q), bits(k), bits(v), plv, ids, counts, ops0, s, sel)
+    same = oracle.attention(bits(q), bits(k), bits(v), pl0, ids0, cnt0, ops0, s, sel)
+    assert pl0.R == plv.R and np.array_equal(base, same)
+    P = 100
+    plv, pl, q, k, v, ops, ids, counts, ids_x, cnt_x = _prefix_case(rng, P, (3, 2, 1), d)
+    Rp = pl.R - plv.R
+    assert Rp == 2
+    assert np.array_equal(cnt_x[0, :plv.R, :2], counts[0, :, :2])
+    assert (cnt_x[0, :plv.R, 2] == counts[0, :, 2] + Rp).all()
+    for a in range(plv.R):
+        n = int(cnt_x[0, a].sum())
+        assert ids_x[0, a, n - Rp:n].tolist() == [plv.R, plv.R + 1]
+    for (a, ju) in ((0, 0), (3, 17)):
+        dbg = oracle.attention_row_debug(bits(q), bits(k), bits(v), pl, ids_x, cnt_x, ops, s, 0, a, ju)
+        kept = ~np.isnan(dbg["shat"])
+        assert kept[:P].all() and kept.sum() == P + sum(int(plv.n_valid[b]) for b in ids[0, a, :6])
+        assert (dbg["tier"][:P] == 16).all()
+        hf = dbg["h_final"]
+        what_fin = np.where(kept, dbg["what"] * np.exp(np.where(kept, dbg["h_at"], 0) - hf), 0.0)
+        o_rec = (what_fin[:, None] * dbg["vhat"]).sum(0) / dbg["ell"]
+        assert np.abs(o_rec - dbg["out"]).max() <= 2.0 ** -8 * max(1.0, np.abs(o_rec).max())
+
+
 def test_prop_3_4_bound_difference_identity():
     """Prop. 3.4: B_v2 - B_v1 = -2 Vmax tau + (tau8 eps8 + tau4 eps4)/(1 - delta_v2)."""
     rng = np.random.default_rng(18)
