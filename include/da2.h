@@ -9,8 +9,9 @@
  *                     online-softmax state and one output accumulator          (Sec. 3.3, App. C.4)
  *
  * Conventions
- *   - q, k, v, out: DEVICE pointers, contiguous bf16 [B, H, N, head_dim], N = T*Hg*Wg, raster token order
- *     u = (t*Hg + y)*Wg + x, 16-byte aligned.  out must not alias the inputs.
+ *   - q, k, v, out: DEVICE pointers, contiguous bf16 [B, H, P + N, head_dim]: first the P = n_prefix prefix (text)
+ *     tokens, if any, then the N = T*Hg*Wg video tokens in raster order u = (t*Hg + y)*Wg + x; 16-byte aligned.
+ *     out must not alias the inputs.
  *   - workspace: DEVICE pointer, 256-byte aligned, at least da2_plan_info().workspace_bytes long.  The caller owns
  *     all device memory; the library allocates none and keeps no device state between calls (one exception:
  *     da2_draft_map_noalloc, which owns a fixed scratch array, see there).
@@ -56,7 +57,11 @@ typedef struct {
   float lambda;                      /* weight of the max-pooled draft branch in [0,1] (Def. 3.1) */
   float softmax_scale;               /* <= 0 selects 1/sqrt(head_dim) */
   int32_t rank_scope;                /* da2_rank_scope_t */
-  int32_t reserved;                  /* must be 0 */
+  int32_t n_prefix;                  /* P >= 0 prefix (text) tokens in front of the video tokens (App. C.1: prefix
+                                        interactions lie outside the region budget).  Every video query keeps all
+                                        prefix keys and every prefix query attends to all keys, both in the 16-bit
+                                        tier; prefix tokens form ceil(P/64) blocks numbered after the video regions.
+                                        Needs rank_scope = DA2_RANK_ROW.  0 = no prefix */
   const float *g_q, *g_k, *g_v;      /* optional HOST arrays [B*H]: NVFP4 per-tensor scales (App. C.3, g_X); NULL =
                                         derived per head as amax/2688.  Copied into the plan. */
 } da2_config_t;
@@ -91,6 +96,11 @@ typedef struct {
   uint32_t qrec_bytes[3], kvrec_bytes[3];
   uint64_t off_dq8, off_dk8;         /* fp32[BH][R]: INT8 block scales of Q and K */
   uint64_t off_dv8;                  /* fp32[BH][d]: E4M3 per-channel scale of V */
+  int32_t n_prefix, R_prefix;        /* prefix tokens and their blocks, ceil(n_prefix / 64); with a prefix, rows and
+                                        blocks R .. R + R_prefix - 1 are the prefix's: counts is int32[BH][R +
+                                        R_prefix][4], the 16-bit records cover R + R_prefix blocks per head, and
+                                        tier_active[2] is set */
+  int32_t row_stride;                /* ROW scope: id entries reserved per video row (its offset is row * row_stride) */
   uint64_t off_order;                /* uint16[BH][2*ceil(R/2)]: query blocks of a head by decreasing list length
                                         (ties: lower index first; 0xFFFF pads an odd R), written in HEAD scope only
                                         (per-row budgets: equal lengths, blocks 2p and 2p+1).  Scheduling only: the

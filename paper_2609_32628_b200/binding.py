@@ -25,7 +25,7 @@ class _Config(ctypes.Structure):
                 ("Wg", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("tile_h", ctypes.c_int32),
                 ("tile_w", ctypes.c_int32), ("frac16", ctypes.c_double), ("frac8", ctypes.c_double),
                 ("frac4", ctypes.c_double), ("lambda_", ctypes.c_float), ("softmax_scale", ctypes.c_float),
-                ("rank_scope", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("rank_scope", ctypes.c_int32), ("n_prefix", ctypes.c_int32),
                 ("g_q", ctypes.POINTER(ctypes.c_float)), ("g_k", ctypes.POINTER(ctypes.c_float)),
                 ("g_v", ctypes.POINTER(ctypes.c_float))]
 
@@ -44,7 +44,8 @@ class PlanInfo(ctypes.Structure):
                 ("off_ids", ctypes.c_uint64), ("off_select", ctypes.c_uint64), ("off_qrec", ctypes.c_uint64 * 3),
                 ("off_kvrec", ctypes.c_uint64 * 3), ("qrec_bytes", ctypes.c_uint32 * 3),
                 ("kvrec_bytes", ctypes.c_uint32 * 3), ("off_dq8", ctypes.c_uint64), ("off_dk8", ctypes.c_uint64),
-                ("off_dv8", ctypes.c_uint64), ("off_order", ctypes.c_uint64)]
+                ("off_dv8", ctypes.c_uint64), ("n_prefix", ctypes.c_int32), ("R_prefix", ctypes.c_int32),
+                ("row_stride", ctypes.c_int32), ("off_order", ctypes.c_uint64)]
 
 
 def load_library():
@@ -107,8 +108,9 @@ class Plan:
 
 def da2_plan(B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float, frac4: float,
              lam: float = 0.2, softmax_scale: float = 0.0, rank_scope: int = DA2_RANK_ROW,
-             g_q=None, g_k=None, g_v=None, tile_h: int = 8, tile_w: int = 8) -> Plan:
-    cfg = _Config(B, H, T, Hg, Wg, head_dim, tile_h, tile_w, frac16, frac8, frac4, lam, softmax_scale, rank_scope, 0,
+             g_q=None, g_k=None, g_v=None, tile_h: int = 8, tile_w: int = 8, n_prefix: int = 0) -> Plan:
+    cfg = _Config(B, H, T, Hg, Wg, head_dim, tile_h, tile_w, frac16, frac8, frac4, lam, softmax_scale, rank_scope,
+                  n_prefix,
                   None, None, None)
     keep = []
     for name, arr in (("g_q", g_q), ("g_k", g_k), ("g_v", g_v)):

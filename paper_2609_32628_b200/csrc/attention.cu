@@ -239,11 +239,11 @@ struct StreamInfo {
 
 __device__ __forceinline__ StreamInfo load_stream(const Params &p, int bh, int a) {
   StreamInfo st;
-  st.a = a < p.R ? a : -1;
+  st.a = a < p.Rt ? a : -1;
   st.n4 = st.n48 = st.L = 0;
   st.ids = nullptr;
-  if (a < p.R) {
-    const int4 c = *reinterpret_cast<const int4 *>(p.counts + ((size_t)bh * p.R + a) * 4);
+  if (a < p.Rt) {
+    const int4 c = *reinterpret_cast<const int4 *>(p.counts + ((size_t)bh * p.Rt + a) * 4);
     st.n4 = c.x; st.n48 = c.x + c.y; st.L = c.x + c.y + c.z;
     st.ids = p.ids + (size_t)bh * p.ids_per_head + c.w;
   }
@@ -262,9 +262,9 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
-  const int R = p.R, pairs = (R + 1) / 2;
+  const int R = p.R, Rt = p.Rt, pairs = (Rt + 1) / 2;
   const int bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
-  __nv_bfloat16 *out_head = out + (size_t)bh * p.N * D;
+  __nv_bfloat16 *out_head = out + (size_t)bh * p.Ntot * D;
   // the two query blocks of this CTA: equally long rows of the head (scheduling order written with the lists)
   int a0 = 2 * pr, a1 = 2 * pr + 1;
   if (ORDERED) {
@@ -345,14 +345,14 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         tc::mbar_arrive_expect_tx(bar(s, B_Q), bytes);
         for (int t = 0; t < 3; ++t)
           if (nn[t] > 0)
-            tc::bulk_g2s(smem + sm.q[s][t], p.qrec[t] + ((size_t)bh * R + S.a) * p.qrec_bytes[t], p.qrec_bytes[t],
+            tc::bulk_g2s(smem + sm.q[s][t], p.qrec[t] + ((size_t)bh * rec_blocks(p, t) + S.a) * p.qrec_bytes[t], p.qrec_bytes[t],
                          bar(s, B_Q));
       }
       __syncwarp();
       const size_t head_blocks = (size_t)bh * R;
       auto list_id = [&](int idx) -> int {
         int b = idx < S.L ? (int)S.ids[idx] : 0;
-        if (b >= R) { atomicExch(p.status, kDevBadList); b = 0; }
+        if (b >= Rt) { atomicExch(p.status, kDevBadList); b = 0; }
         return b;
       };
       auto key_scale = [&](int idx, int b) -> float {
@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       };
       auto record = [&](int idx, int b) -> unsigned long long {
         const int t = S.tier(idx);
-        return reinterpret_cast<unsigned long long>(p.kvrec[t] + (head_blocks + b) * p.kvrec_bytes[t]);
+        return reinterpret_cast<unsigned long long>(p.kvrec[t] + ((size_t)bh * rec_blocks(p, t) + b) * p.kvrec_bytes[t]);
       };
       int nxt_b = list_id(32 + lane), nn_b = list_id(64 + lane);
       float cur_dk, nxt_dk = key_scale(32 + lane, nxt_b);
@@ -535,7 +535,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     const StreamInfo S = s ? st1 : st0;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const float gqk = p.gscale[bh * 4 + 0] * p.gscale[bh * 4 + 1] * p.scale * kLog2e;
-    const float dq8s = (S.a >= 0 && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
+    const float dq8s = (S.a >= 0 && S.a < R && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
     const float c16 = p.scale * kLog2e;
     float h_own = -INFINITY, ell = 0.f;  // log2-domain maximum after this warp's last step; its partial denominator
     const int g = par;                   // buffers of this warp's step parity
@@ -882,7 +882,7 @@ cudaError_t launch_bounded_wait_probe(int *status, long long limit_cycles, cudaS
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches) {
   const SmemMap sm = make_smem_map(p);
   cudaError_t e;
-  const int grid = p.BH * ((p.R + 1) / 2);
+  const int grid = p.BH * ((p.Rt + 1) / 2);
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
     if (err != cudaSuccess) return err;

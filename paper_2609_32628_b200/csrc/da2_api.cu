@@ -39,6 +39,8 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
   std::memset(&p, 0, sizeof(p));
   p.B = I.B; p.H = I.H; p.T = I.T; p.Hg = I.Hg; p.Wg = I.Wg; p.d = I.head_dim;
   p.nty = I.nty; p.ntx = I.ntx; p.R_f = I.R_f; p.R = I.R; p.N = I.N; p.BH = I.B * I.H;
+  p.P = I.n_prefix; p.Rp = I.R_prefix; p.Rt = I.R + I.R_prefix; p.Ntot = I.N + I.n_prefix;
+  p.row_stride = I.row_stride;
   p.rank_scope = I.rank_scope;
   for (int t = 0; t < 3; ++t) {
     p.tier_active[t] = I.tier_active[t];
@@ -98,7 +100,9 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
     return DA2_ERR_INVALID_ARG;
   if (!(cfg->lambda >= 0.0f && cfg->lambda <= 1.0f)) return DA2_ERR_INVALID_ARG;
   if (cfg->rank_scope != DA2_RANK_ROW && cfg->rank_scope != DA2_RANK_HEAD) return DA2_ERR_INVALID_ARG;
-  if (cfg->reserved != 0) return DA2_ERR_INVALID_ARG;
+  if (cfg->n_prefix < 0 || cfg->n_prefix > (1 << 20)) return DA2_ERR_INVALID_ARG;
+  // prefix rows need a list layout with per-row offsets that the head-level ranking does not reserve room for
+  if (cfg->n_prefix > 0 && cfg->rank_scope == DA2_RANK_HEAD) return DA2_ERR_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return DA2_ERR_UNSUPPORTED;
   if (cfg->tile_h != 8 || cfg->tile_w != 8) return DA2_ERR_UNSUPPORTED;
 
@@ -116,6 +120,10 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   I.R_f = I.nty * I.ntx;
   long long R = (long long)cfg->T * I.R_f;
   if (R > 16384) { delete plan; return DA2_ERR_UNSUPPORTED; }  // ids are uint16; row buffers live in shared memory
+  const long long Rp = ((long long)cfg->n_prefix + da2::kSlots - 1) / da2::kSlots, Rt = R + Rp;
+  if (Rt > 65535) { delete plan; return DA2_ERR_UNSUPPORTED; }
+  I.n_prefix = cfg->n_prefix;
+  I.R_prefix = (int32_t)Rp;
   I.R = (int32_t)R;
   I.S = da2::kSlots;
   I.N = (int64_t)cfg->T * cfg->Hg * cfg->Wg;
@@ -126,14 +134,17 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   long long qt[3];
   quotas_from_fractions(cfg->frac16, cfg->frac8, cfg->frac4, M, qt);
   for (int t = 0; t < 3; ++t) { I.quota[t] = qt[t]; I.tier_active[t] = qt[t] > 0; }
+  if (Rp > 0) I.tier_active[2] = 1;  // prefix interactions run in the 16-bit tier, outside the budget
 
   const uint64_t BH = (uint64_t)cfg->B * cfg->H, d = cfg->head_dim, S = da2::kSlots;
   const long long kept = qt[0] + qt[1] + qt[2];
   if (cfg->rank_scope == DA2_RANK_ROW) {
-    long long stride = (kept + 7) / 8 * 8;
+    long long stride = (kept + Rp + 7) / 8 * 8;
     if (stride == 0) stride = 8;
-    I.ids_per_head = stride * R;
+    I.row_stride = (int32_t)stride;
+    I.ids_per_head = stride * R + Rp * ((Rt + 7) / 8 * 8);  // video rows, then the prefix rows (every block each)
   } else {
+    I.row_stride = 0;
     I.ids_per_head = (kept + 7) / 8 * 8 + 8;
   }
 
@@ -153,12 +164,13 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   for (int i = 0; i < 4; ++i) I.off_desc[i] = c.take(BH * R * d * 4);
   for (int i = 0; i < 2; ++i) I.off_logits[i] = c.take(BH * R * R * 4);
   I.off_map = c.take(BH * R * R * 4);
-  I.off_counts = c.take(BH * R * 4 * 4);
+  I.off_counts = c.take(BH * (uint64_t)Rt * 4 * 4);
   I.off_ids = c.take(BH * (uint64_t)I.ids_per_head * 2);
   I.off_select = c.take(BH * (4096 + 8 * (uint64_t)R) * 4);
   for (int t = 0; t < 3; ++t) {
-    I.off_qrec[t] = c.take(I.tier_active[t] ? BH * R * I.qrec_bytes[t] : 0);
-    I.off_kvrec[t] = c.take(I.tier_active[t] ? BH * R * I.kvrec_bytes[t] : 0);
+    const uint64_t blocks = t == 2 ? (uint64_t)Rt : (uint64_t)R;  // the 16-bit tier also holds the prefix blocks
+    I.off_qrec[t] = c.take(I.tier_active[t] ? BH * blocks * I.qrec_bytes[t] : 0);
+    I.off_kvrec[t] = c.take(I.tier_active[t] ? BH * blocks * I.kvrec_bytes[t] : 0);
   }
   I.off_dq8 = c.take(BH * R * 4);
   I.off_dk8 = c.take(BH * R * 4);
@@ -222,6 +234,7 @@ da2_status_t prepare_impl(const da2_plan_t *plan, const void *q, const void *k, 
   if (select) {
     if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (da2::launch_prefix_rows(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     // rows of unequal length (HEAD scope) are paired by length; with per-row budgets the order is the identity
     if (plan->info.rank_scope != 0 && da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   }
@@ -260,6 +273,7 @@ da2_status_t da2_prepare_cached_scales(const da2_plan_t *plan, const void *q, co
   if (reselect) {
     if (da2::launch_draft(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     if (da2::launch_rank(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
+    if (da2::launch_prefix_rows(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
     if (plan->info.rank_scope != 0 && da2::launch_order(p, st, &launches) != cudaSuccess) return DA2_ERR_CUDA;
   }
   t_last_launches = launches;

@@ -22,7 +22,10 @@ constexpr int kDevBadList = 2;
 struct Params {
   int B, H, T, Hg, Wg, d;
   int nty, ntx, R_f, R;
-  long long N;
+  long long N;              // video tokens per head
+  int P, Rp, Rt;            // prefix tokens, prefix blocks (ceil(P / 64)), blocks per head R + Rp
+  long long Ntot;           // tokens per head in the tensors: P prefix tokens, then the N video tokens
+  int row_stride;           // id entries reserved per video row (ROW scope)
   int BH;
   int rank_scope;
   int tier_active[3];       // 0: NVFP4, 1: INT8/E4M3, 2: BF16
@@ -47,7 +50,12 @@ struct Params {
 };
 
 // number of valid rows / columns of tile (ty, tx) and the 64-bit slot-valid mask of block a
+// (blocks R .. R + Rp - 1 are runs of 64 consecutive prefix tokens; the last one may be short)
 __host__ __device__ inline unsigned long long block_valid_mask(const Params &p, int a) {
+  if (a >= p.R) {
+    const int rem = p.P - (a - p.R) * kSlots;
+    return rem >= kSlots ? ~0ull : ((1ull << rem) - 1ull);
+  }
   int r = a % p.R_f;
   int ty = r / p.ntx, tx = r % p.ntx;
   int vr = min(kTile, p.Hg - ty * kTile), vc = min(kTile, p.Wg - tx * kTile);
@@ -57,13 +65,18 @@ __host__ __device__ inline unsigned long long block_valid_mask(const Params &p, 
   return m;
 }
 
-// raster token index of slot j of block a (caller checks validity with the mask)
+// token index (row of a head's [P + N, d] tensor) of slot j of block a: prefix tokens come first, then the video
+// tokens in raster order (caller checks validity with the mask)
 __host__ __device__ inline long long slot_token(const Params &p, int a, int j) {
+  if (a >= p.R) return (long long)(a - p.R) * kSlots + j;
   int t = a / p.R_f, r = a % p.R_f;
   int ty = r / p.ntx, tx = r % p.ntx;
   int y = ty * kTile + (j >> 3), x = tx * kTile + (j & 7);
-  return ((long long)t * p.Hg + y) * p.Wg + x;
+  return p.P + ((long long)t * p.Hg + y) * p.Wg + x;
 }
+
+// operand records per head and tier: the 16-bit tier also holds the prefix blocks
+__host__ __device__ inline int rec_blocks(const Params &p, int tier) { return tier == 2 ? p.Rt : p.R; }
 
 // kernel launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_pool(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
@@ -72,6 +85,7 @@ cudaError_t launch_draft(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_rank(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_map_rows(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_order(const Params &p, cudaStream_t st, int *launches);
+cudaError_t launch_prefix_rows(const Params &p, cudaStream_t st, int *launches);
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches, bool pool = false);
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);

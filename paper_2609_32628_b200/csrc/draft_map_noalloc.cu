@@ -58,7 +58,7 @@ extern "C" da2_status_t da2_draft_map_noalloc(const float *q_avg, const float *q
   if (scratch_address(&scratch) != cudaSuccess) return DA2_ERR_CUDA;
 
   da2::Params p = {};
-  p.BH = BH; p.B = BH; p.H = 1; p.R = R; p.d = head_dim;
+  p.BH = BH; p.B = BH; p.H = 1; p.R = R; p.Rt = R; p.d = head_dim;
   p.lambda = lambda;
   p.scale = softmax_scale;
   p.desc[0] = const_cast<float *>(q_avg);

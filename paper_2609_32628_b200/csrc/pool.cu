@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(256) pool_kernel(Params p, const __nv_bfloat16
   const int cidx = tid % CPR, tsub = tid / CPR;
   const unsigned long long mask = block_valid_mask(p, a);
   const int n_valid = __popcll(mask);
-  const size_t head_off = (size_t)bh * p.N * D;
+  const size_t head_off = (size_t)bh * p.Ntot * D;
 
   double sq[8], sk[8];
   float mq[8], mk[8], av[8];

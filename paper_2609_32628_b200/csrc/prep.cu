@@ -71,8 +71,10 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 
   const int a = blockIdx.x, bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long mask = block_valid_mask(p, a);
-  const size_t head_off = (size_t)bh * p.N * D;
-  const size_t blk = (size_t)bh * p.R + a;
+  const size_t head_off = (size_t)bh * p.Ntot * D;
+  const size_t blk = (size_t)bh * p.R + a;        // record index in the quantised tiers (video blocks only)
+  const size_t blk16 = (size_t)bh * p.Rt + a;     // record index in the 16-bit tier (video and prefix blocks)
+  const bool video = a < p.R;                      // prefix blocks only ever run in the 16-bit tier (App. C.1)
 
   // stage the three tiles, padding slots as zeros; track max|Q|, max|K| of the block
   float aq = 0.f, ak = 0.f;
@@ -109,11 +111,11 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
     for (int w = 0; w < NT / 32; ++w) m = fmaxf(m, s_red[tid][w]);
     const float delta = __fadd_rn(__fdiv_rn(m, 127.0f), 1e-7f);
     s_delta[tid] = delta;
-    if (p.tier_active[1]) (tid == 0 ? p.dq8 : p.dk8)[blk] = delta;
+    if (p.tier_active[1] && video) (tid == 0 ? p.dq8 : p.dk8)[blk] = delta;
   }
   __syncthreads();
 
-  if (POOL) {
+  if (POOL && video) {
     // one thread per (tensor, channel): sum and maximum over the valid slots of the staged tile.  A sum of at most
     // 64 bf16 values is exact in fp64, so the mean is correctly rounded whatever the order.
     const int n_valid = __popcll(mask);
@@ -137,8 +139,8 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 
   // ------------------------------------------------------------------ tier 2: BF16, reorder only
   if (p.tier_active[2]) {
-    uint8_t *qr = p.qrec[2] + blk * p.qrec_bytes[2];
-    uint8_t *kr = p.kvrec[2] + blk * p.kvrec_bytes[2];
+    uint8_t *qr = p.qrec[2] + blk16 * p.qrec_bytes[2];
+    uint8_t *kr = p.kvrec[2] + blk16 * p.kvrec_bytes[2];
     uint8_t *vr = kr + kSlots * D * 2;
     for (int idx = tid; idx < kSlots * D / 8; idx += NT) {  // chunk (kc, r): channels kc*8.. of slot r
       const int kc = idx / kSlots, r = idx % kSlots;
@@ -156,7 +158,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
   }
 
   // ------------------------------------------------------------------ tier 1: INT8 Q/K, E4M3 V
-  if (p.tier_active[1]) {
+  if (p.tier_active[1] && video) {
     uint8_t *qr = p.qrec[1] + blk * p.qrec_bytes[1];
     uint8_t *kr = p.kvrec[1] + blk * p.kvrec_bytes[1];
     uint8_t *vr = kr + kSlots * D;
@@ -192,7 +194,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
   }
 
   // ------------------------------------------------------------------ tier 0: NVFP4
-  if (p.tier_active[0]) {
+  if (p.tier_active[0] && video) {
     const float gq = p.gscale[bh * 4 + 0], gk = p.gscale[bh * 4 + 1], gv = p.gscale[bh * 4 + 2];
     constexpr int QK_IMG = kSlots * D / 2, NATOM = D / 64;
     uint8_t *qr = p.qrec[0] + blk * p.qrec_bytes[0];
@@ -256,7 +258,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches, bool pool) {
-  dim3 grid(p.R, p.BH);
+  dim3 grid(p.Rt, p.BH);
   const size_t smem = 3 * (size_t)kSlots * p.d * 2 + 3 * kSfAtomBytes;
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(NT) rank_row_kernel(Params p) {
   }
   int pos[3] = {cnt[0], cnt[1], cnt[2]};
   block_scan<3>(pos, tot, scratch);
-  const int stride = (int)(p.ids_per_head / R);
+  const int stride = p.row_stride;
   uint16_t *ids = p.ids + (size_t)bh * p.ids_per_head + (size_t)a * stride;
   const int base[3] = {0, tot[0], tot[0] + tot[1]};
   {
@@ -222,9 +222,24 @@ __global__ void __launch_bounds__(NT) rank_row_kernel(Params p) {
       for (int t = 0; t < 3; ++t) er[t] += key == bd[t].value;
     }
   }
+  // prefix interactions lie outside the budget: every video row keeps all prefix blocks, in the 16-bit segment
+  for (int j = threadIdx.x; j < p.Rp; j += NT) ids[tot[0] + tot[1] + tot[2] + j] = (uint16_t)(R + j);
   if (threadIdx.x == 0) {
-    int *c = p.counts + ((size_t)bh * R + a) * 4;
-    c[0] = tot[0]; c[1] = tot[1]; c[2] = tot[2]; c[3] = a * stride;
+    int *c = p.counts + ((size_t)bh * p.Rt + a) * 4;
+    c[0] = tot[0]; c[1] = tot[1]; c[2] = tot[2] + p.Rp; c[3] = a * stride;
+  }
+}
+
+// Prefix query rows are not sparse (App. C.1): their list is every block of the head, video and prefix, 16-bit.
+__global__ void __launch_bounds__(NT) prefix_rows_kernel(Params p) {
+  const int j = blockIdx.x, bh = blockIdx.y, a = p.R + j;
+  const int pstride = (p.Rt + 7) / 8 * 8;
+  const int off = p.R * p.row_stride + j * pstride;
+  uint16_t *ids = p.ids + (size_t)bh * p.ids_per_head + off;
+  for (int b = threadIdx.x; b < p.Rt; b += NT) ids[b] = (uint16_t)b;
+  if (threadIdx.x == 0) {
+    int *c = p.counts + ((size_t)bh * p.Rt + a) * 4;
+    c[0] = 0; c[1] = 0; c[2] = p.Rt; c[3] = off;
   }
 }
 
@@ -471,6 +486,13 @@ __global__ void __launch_bounds__(256) order_rows_kernel(Params p) {
   }
 }
 }  // namespace
+
+cudaError_t launch_prefix_rows(const Params &p, cudaStream_t st, int *launches) {
+  if (p.Rp == 0) return cudaSuccess;
+  prefix_rows_kernel<<<dim3(p.Rp, p.BH), NT, 0, st>>>(p);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_order(const Params &p, cudaStream_t st, int *launches) {
   const size_t smem = (size_t)p.R * sizeof(int);
