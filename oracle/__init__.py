@@ -43,6 +43,7 @@ def lib():
         _lib.orc_cast_e2m1.restype = ctypes.c_uint8
         _lib.orc_cast_e2m1.argtypes = [ctypes.c_float]
         _lib.orc_plan.restype = ctypes.c_int
+        _lib.orc_plan_balanced.restype = ctypes.c_int
     return _lib
 
 
@@ -122,6 +123,19 @@ def plan(T: int, Hg: int, Wg: int, th: int = 8, tw: int = 8) -> Plan:
     nv = np.empty((R,), np.int32)
     lib().orc_plan(_i(T), _i(Hg), _i(Wg), _i(th), _i(tw), _p(st), _p(nv))
     return Plan(T, Hg, Wg, th, tw, R, S, st, nv)
+
+
+def plan_balanced(T: int, Hg: int, Wg: int, C: int = 64) -> Plan:
+    """Balanced ragged minimum-perimeter partition (App. C.2): R_f = ceil(Hg*Wg/C) connected regions per frame whose
+    sizes differ by at most one; .choice = (transposed, bands, perimeter of one frame)."""
+    R = lib().orc_plan_balanced(_i(T), _i(Hg), _i(Wg), _i(C), None, None, None)
+    st = np.empty((R, C), np.int32)
+    nv = np.empty((R,), np.int32)
+    choice = (ctypes.c_int64 * 3)()
+    lib().orc_plan_balanced(_i(T), _i(Hg), _i(Wg), _i(C), _p(st), _p(nv), choice)
+    pl = Plan(T, Hg, Wg, 0, 0, R, C, st, nv, 0, R)
+    pl.choice = (int(choice[0]), int(choice[1]), int(choice[2]))
+    return pl
 
 
 # ---------------------------------------------------------------- prefix tokens

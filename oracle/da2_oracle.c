@@ -126,6 +126,104 @@ int orc_plan(int T, int Hg, int Wg, int th, int tw, int32_t *slot_token, int32_t
   return R;
 }
 
+/* ------------------------------------------------- balanced ragged partition (App. C.2)
+ * Every H x W frame is cut into R_f = ceil(HW / C) connected regions of balanced size (sizes differ by at
+ * most one, so padding is below one block per frame, Eq. "ragged-padding"), and among candidate partitions
+ * the one with the smallest total perimeter is taken (Eq. "region-perimeter").  The paper names neither the
+ * candidates nor the order of tokens inside a block; this reading fixes both:
+ *   - a candidate is a band order: the frame is cut into r bands along one axis (heights as equal as
+ *     possible, the taller ones first); bands are walked one after the other, band b column by column
+ *     (left to right for even b, right to left for odd b), the columns alternately downwards and upwards,
+ *     the first column of every band downwards; "transposed" candidates do the same with rows and columns
+ *     exchanged.  Cutting that order into R_f consecutive runs, the first HW mod R_f of them one token
+ *     longer, gives the regions; slot j of a block is the j-th token of its run.
+ *   - a candidate is admissible if every region is 4-connected; the admissible candidate with the smallest
+ *     total perimeter wins, ties going to bands along rows first and then to fewer bands.  r = H (rows as
+ *     bands) is always admissible, so a winner exists. */
+static void band_order(int H, int W, int r, int transposed, int32_t *order /* [H*W] cell = y*W+x */) {
+  int L = transposed ? W : H, M = transposed ? H : W; /* bands cut the axis of length L, columns run along M */
+  int hb = L / r, extra = L % r, pos = 0, l0 = 0;
+  for (int b = 0; b < r; ++b) {
+    int h = hb + (b < extra);
+    for (int i = 0; i < M; ++i) {
+      int m = (b % 2 == 0) ? i : M - 1 - i;
+      for (int k = 0; k < h; ++k) {
+        int l = l0 + ((i % 2 == 0) ? k : h - 1 - k);
+        order[pos++] = transposed ? (m * W + l) : (l * W + m);
+      }
+    }
+    l0 += h;
+  }
+}
+
+static int regions_connected(int H, int W, int Rf, const int32_t *region /* [H*W] */, int32_t *stack, uint8_t *seen) {
+  for (int i = 0; i < H * W; ++i) seen[i] = 0;
+  int comps = 0;
+  for (int c0 = 0; c0 < H * W; ++c0) {
+    if (seen[c0]) continue;
+    ++comps;
+    int top = 0;
+    stack[top++] = c0;
+    seen[c0] = 1;
+    while (top) {
+      int c = stack[--top], y = c / W, x = c % W;
+      const int ny[4] = {y - 1, y + 1, y, y}, nx[4] = {x, x, x - 1, x + 1};
+      for (int e = 0; e < 4; ++e) {
+        if (ny[e] < 0 || ny[e] >= H || nx[e] < 0 || nx[e] >= W) continue;
+        int c2 = ny[e] * W + nx[e];
+        if (!seen[c2] && region[c2] == region[c]) { seen[c2] = 1; stack[top++] = c2; }
+      }
+    }
+  }
+  return comps == Rf;
+}
+
+static i64 total_perimeter(int H, int W, const int32_t *region) {
+  i64 per = 0;
+  for (int y = 0; y < H; ++y)
+    for (int x = 0; x < W; ++x) {
+      int c = y * W + x;
+      per += (y == 0) + (y == H - 1) + (x == 0) + (x == W - 1);
+      if (y + 1 < H && region[c + W] != region[c]) per += 2;
+      if (x + 1 < W && region[c + 1] != region[c]) per += 2;
+    }
+  return per;
+}
+
+/* Returns R = T * R_f.  slot_token: [R*C] (-1 = padding), n_valid: [R]; choice[0..2] = (transposed, bands,
+ * total perimeter of one frame).  Outputs may be NULL. */
+int orc_plan_balanced(int T, int Hg, int Wg, int C, int32_t *slot_token, int32_t *n_valid, i64 *choice) {
+  int HW = Hg * Wg, Rf = (HW + C - 1) / C, n = HW / Rf, rem = HW % Rf;
+  int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)HW), *best = (int32_t *)malloc(sizeof(int32_t) * (size_t)HW);
+  int32_t *region = (int32_t *)malloc(sizeof(int32_t) * (size_t)HW), *stack = (int32_t *)malloc(sizeof(int32_t) * (size_t)HW);
+  uint8_t *seen = (uint8_t *)malloc((size_t)HW);
+  i64 best_per = -1;
+  int best_t = 0, best_r = 0;
+  for (int tr = 0; tr < 2; ++tr)
+    for (int r = 1; r <= (tr ? Wg : Hg); ++r) {
+      band_order(Hg, Wg, r, tr, order);
+      for (int a = 0, pos = 0; a < Rf; ++a)
+        for (int j = 0; j < n + (a < rem); ++j) region[order[pos++]] = a;
+      if (!regions_connected(Hg, Wg, Rf, region, stack, seen)) continue;
+      i64 per = total_perimeter(Hg, Wg, region);
+      if (best_per < 0 || per < best_per) {
+        best_per = per; best_t = tr; best_r = r;
+        for (int i = 0; i < HW; ++i) best[i] = order[i];
+      }
+    }
+  if (choice) { choice[0] = best_t; choice[1] = best_r; choice[2] = best_per; }
+  for (int t = 0; t < T; ++t)
+    for (int a = 0, pos = 0; a < Rf; ++a) {
+      int na = n + (a < rem);
+      for (int j = 0; j < C; ++j)
+        if (slot_token) slot_token[((i64)t * Rf + a) * C + j] = j < na ? t * HW + best[pos + j] : -1;
+      if (n_valid) n_valid[t * Rf + a] = na;
+      pos += na;
+    }
+  free(order); free(best); free(region); free(stack); free(seen);
+  return T * Rf;
+}
+
 /* Integer quotas from fractions of M candidates: cumulative round-half-up, so the
  * three counts always sum to round(sum of fractions * M) (App. C.1: integer quotas
  * T_p with sum T; the rounding rule is this implementation's reading). */

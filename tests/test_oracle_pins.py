@@ -72,6 +72,137 @@ def test_plan_perimeter_identity(grid):
     assert per == 2 * (Hg + Wg) + 2 * cut
 
 
+def _frame_regions(pl, Hg, Wg):
+    """Region id of every cell of frame 0, from the slot table."""
+    Rf = pl.R // pl.T
+    region = np.full(Hg * Wg, -1)
+    for a in range(Rf):
+        toks = pl.slot_token[a][pl.slot_token[a] >= 0]
+        assert (region[toks] == -1).all()
+        region[toks] = a
+    assert (region >= 0).all()
+    return region.reshape(Hg, Wg), Rf
+
+
+def _perimeter_by_edges(region):
+    """Sum over regions of their unit boundary edges, counted cell by cell."""
+    H, W = region.shape
+    per = 0
+    cut = 0
+    for y in range(H):
+        for x in range(W):
+            for dy, dx in ((0, 1), (1, 0), (0, -1), (-1, 0)):
+                yy, xx = y + dy, x + dx
+                if not (0 <= yy < H and 0 <= xx < W):
+                    per += 1
+                elif region[yy, xx] != region[y, x]:
+                    per += 1
+                    cut += 1
+    return per, cut // 2
+
+
+@pytest.mark.parametrize("grid", [(2, 30, 52), (1, 45, 80), (3, 12, 20), (1, 9, 13), (1, 32, 32), (1, 7, 5)])
+@pytest.mark.parametrize("C", [64, 128])
+def test_balanced_partition_invariants(grid, C):
+    """App. C.2: R_f = ceil(HW / C) regions per frame, less than one block of padding per frame
+    (Eq. 'ragged-padding'), balanced sizes, every region connected (scipy's component labelling), the slot table a
+    bijection that repeats frame by frame, and Eq. 'region-perimeter' by brute-force edge count."""
+    from scipy import ndimage
+    T, Hg, Wg = grid
+    pl = oracle.plan_balanced(T, Hg, Wg, C)
+    HW = Hg * Wg
+    Rf = -(-HW // C)
+    assert pl.R == T * Rf and pl.S == C
+    assert 0 <= Rf * C - HW < C
+    assert int(pl.n_valid.sum()) == T * HW and pl.n_valid.max() - pl.n_valid.min() <= 1 and pl.n_valid.max() <= C
+    toks = pl.slot_token[pl.slot_token >= 0]
+    assert np.array_equal(np.sort(toks), np.arange(T * HW))
+    for a in range(pl.R):   # valid slots come first, padding after them
+        assert (pl.slot_token[a, :pl.n_valid[a]] >= 0).all() and (pl.slot_token[a, pl.n_valid[a]:] == -1).all()
+    for t in range(1, T):   # the same partition in every frame
+        assert np.array_equal(pl.slot_token[t * Rf:(t + 1) * Rf][pl.slot_token[:Rf] >= 0],
+                              pl.slot_token[:Rf][pl.slot_token[:Rf] >= 0] + t * HW)
+    region, _ = _frame_regions(pl, Hg, Wg)
+    for a in range(Rf):
+        _, ncomp = ndimage.label(region == a)
+        assert ncomp == 1, f"region {a} is not connected"
+    per, cut = _perimeter_by_edges(region)
+    assert per == 2 * (Hg + Wg) + 2 * cut
+    assert pl.choice[2] == per
+    # the winner is no worse than the always-admissible candidate of single-row bands, written out here
+    strips = np.empty(HW, int)
+    order = [y * Wg + (x if y % 2 == 0 else Wg - 1 - x) for y in range(Hg) for x in range(Wg)]
+    n, rem = divmod(HW, Rf)
+    pos = 0
+    for a in range(Rf):
+        for _ in range(n + (a < rem)):
+            strips[order[pos]] = a
+            pos += 1
+    assert per <= _perimeter_by_edges(strips.reshape(Hg, Wg))[0]
+
+
+def test_balanced_partition_against_fixed_tiles_and_exhaustive_search():
+    """(i) Where 8 x 8 tiles divide the frame, the balanced partition of capacity 64 IS the tile partition.
+    (ii) On the 720p latent frame it needs 57 blocks instead of 60 and its perimeter does not exceed the tiles'.
+    (iii) On tiny frames an exhaustive search over ALL partitions into connected regions of the balanced sizes finds
+    no smaller perimeter than the chosen candidate's."""
+    for Hg, Wg in ((16, 16), (32, 48)):
+        a, _ = _frame_regions(oracle.plan_balanced(1, Hg, Wg, 64), Hg, Wg)
+        b, _ = _frame_regions(oracle.plan(1, Hg, Wg), Hg, Wg)
+        # same partition up to the numbering of the regions
+        pairs = set(zip(a.ravel().tolist(), b.ravel().tolist()))
+        assert len(pairs) == a.max() + 1 == b.max() + 1
+    bal, fix = oracle.plan_balanced(1, 45, 80, 64), oracle.plan(1, 45, 80)
+    assert (bal.R, fix.R) == (57, 60)
+    assert bal.choice[2] <= _perimeter_by_edges(_frame_regions(fix, 45, 80)[0])[0]
+
+    def best_perimeter(H, W, sizes):
+        best = [None]
+        grid = [-1] * (H * W)
+
+        def neighbours(c):
+            y, x = divmod(c, W)
+            return [cc for cc, ok in (((y - 1) * W + x, y > 0), ((y + 1) * W + x, y < H - 1),
+                                      (y * W + x - 1, x > 0), (y * W + x + 1, x < W - 1)) if ok]
+
+        def grow(a, cells, frontier_min):
+            if len(cells) == sizes[a]:
+                place(a + 1)
+                return
+            cand = sorted({n for c in cells for n in neighbours(c) if grid[n] == -1 and n > frontier_min})
+            for n in cand:       # canonical growth: only cells above the region's first cell, each set once
+                grid[n] = a
+                grow(a, cells + [n], frontier_min)
+                grid[n] = -1
+            return
+
+        seen = set()
+
+        def place(a):
+            if a == len(sizes):
+                key = tuple(grid)
+                if key in seen:
+                    return
+                seen.add(key)
+                per = _perimeter_by_edges(np.array(grid).reshape(H, W))[0]
+                best[0] = per if best[0] is None else min(best[0], per)
+                return
+            first = grid.index(-1)      # the region that owns the first free cell is placed next
+            grid[first] = a
+            grow(a, [first], first)
+            grid[first] = -1
+
+        place(0)
+        return best[0]
+
+    for (H, W, C) in ((4, 4, 4), (2, 6, 4), (3, 4, 4), (3, 3, 3)):
+        pl = oracle.plan_balanced(1, H, W, C)
+        sizes = sorted(pl.n_valid.tolist(), reverse=True)
+        # the exhaustive search lets any region take any of the balanced sizes: try every ordering of sizes
+        cands = {best_perimeter(H, W, list(p)) for p in set(itertools.permutations(sizes))}
+        assert pl.choice[2] == min(c for c in cands if c is not None), (H, W, C)
+
+
 def test_quotas_match_budget_tables():
     # exact retained-block counts per query-block row for the named workloads
     assert oracle.quotas(0.0, 0.25, 0.25, 16) == (0, 4, 4)
