@@ -83,10 +83,13 @@ def flop_counts(w, plan, ws):
     cnt = ws[I.off_counts:I.off_counts + BH * R * 16].view(torch.int32).view(BH, R, 4).long()
     padded = [float(cnt[:, :, t].sum().item()) * 4 * 64 * 64 * d for t in range(3)]
     # valid tokens per block
-    nty, ntx = I.nty, I.ntx
-    vr = torch.tensor([min(8, w.Hg - 8 * ty) for ty in range(nty)], device=ws.device)
-    vc = torch.tensor([min(8, w.Wg - 8 * tx) for tx in range(ntx)], device=ws.device)
-    nv = (vr[:, None] * vc[None, :]).reshape(-1).repeat(w.T).double()  # [R]
+    if I.partition == 0:
+        nty, ntx = I.nty, I.ntx
+        vr = torch.tensor([min(8, w.Hg - 8 * ty) for ty in range(nty)], device=ws.device)
+        vc = torch.tensor([min(8, w.Wg - 8 * tx) for tx in range(ntx)], device=ws.device)
+        nv = (vr[:, None] * vc[None, :]).reshape(-1).repeat(w.T).double()  # [R]
+    else:   # balanced ragged partition: region r of a frame holds part_n + (r < part_rem) tokens
+        nv = (I.part_n + (torch.arange(I.R_f, device=ws.device) < I.part_rem).long()).repeat(w.T).double()
     valid = [0.0, 0.0, 0.0]
     if I.rank_scope == 0:
         stride = int(I.ids_per_head) // R
@@ -234,7 +237,7 @@ def run_da2(args, rank, world, local_rank):
     w = rank_workload(args.workload, rank)
     q, k, v = da2_inputs.make_qkv(w, dev)
     plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
-                        rank_scope=args.rank_scope)
+                        rank_scope=args.rank_scope, partition=args.partition)
     ws = torch.empty(int(plan.info.workspace_bytes), dtype=torch.uint8, device=dev)
     out = torch.empty_like(q)
     stream = torch.cuda.current_stream()
@@ -320,7 +323,7 @@ def run_da2(args, rank, world, local_rank):
     e2e_serial_ms = timed(serial_step)
     del dq, dk, dv
     pipe = da2.HostPipeline(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
-                            rank_scope=args.rank_scope, groups="ramp", device=dev)
+                            rank_scope=args.rank_scope, groups="ramp", device=dev, partition=args.partition)
     groups = [b - a for a, b in pipe.ranges]
     e2e_ms = timed(lambda: pipe.run(hq, hk, hv, hout))
     assert pipe.status() == 0, "device status after the end-to-end region"
@@ -370,6 +373,7 @@ def run_da2(args, rank, world, local_rank):
         "config": {"workload": args.workload, "B": w.B * world, "H": w.H, "head_dim": w.head_dim,
                    "grid": [w.T, w.Hg, w.Wg], "tokens": w.N, "budget_16_8_4": [w.frac16, w.frac8, w.frac4],
                    "rank_scope": "row" if args.rank_scope == 0 else "head",
+                   "partition": "8x8 tiles" if args.partition == 0 else "balanced ragged, capacity 64",
                    "l2": "inputs larger than L2 (Q, K, V and operand records are several GB per step)"},
         "e2e": {"value": dense * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": out.numel() * 2,
@@ -447,6 +451,8 @@ def main():
     ap.add_argument("--impl", default="da2", choices=["da2", "reference"])
     ap.add_argument("--workload", default="wan14b_720p", choices=sorted(da2_inputs.WORKLOADS))
     ap.add_argument("--rank-scope", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--partition", type=int, default=0, choices=[0, 1],
+                    help="0: fixed 8x8 tiles (the benchmark configurations); 1: balanced ragged partition (App. C.2)")
     ap.add_argument("--cpu-blocks", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mma-peaks", action="store_true",

@@ -50,6 +50,15 @@ typedef enum {
  * Alg. 1, so rows may keep different numbers of blocks, possibly none. */
 typedef enum { DA2_RANK_ROW = 0, DA2_RANK_HEAD = 1 } da2_rank_scope_t;
 
+/* How a latent frame is cut into regions (one region = one block of 64 slots).
+ * TILES: fixed 8 x 8 spatial tiles, ragged edge tiles padded (the benchmark configurations).
+ * BALANCED: the ragged partition of App. C.2: R_f = ceil(Hg*Wg / capacity) connected regions per frame whose token
+ * counts differ by at most one (less than one block of padding per frame, Eq. "ragged-padding"), chosen with the
+ * smallest total perimeter (Eq. "region-perimeter") among band-order candidates: the frame is cut into bands along
+ * one axis, the bands are walked column by column in alternating directions, and that order is cut into R_f runs;
+ * slot j of a block is the j-th token of its run. */
+typedef enum { DA2_PARTITION_TILES = 0, DA2_PARTITION_BALANCED = 1 } da2_partition_t;
+
 typedef struct {
   int32_t B, H, T, Hg, Wg, head_dim; /* head_dim in {64, 128} */
   int32_t tile_h, tile_w;            /* spatial tile of one block; only 8 x 8 is supported */
@@ -64,6 +73,9 @@ typedef struct {
                                         Needs rank_scope = DA2_RANK_ROW.  0 = no prefix */
   const float *g_q, *g_k, *g_v;      /* optional HOST arrays [B*H]: NVFP4 per-tensor scales (App. C.3, g_X); NULL =
                                         derived per head as amax/2688.  Copied into the plan. */
+  int32_t partition;                 /* da2_partition_t */
+  int32_t capacity;                  /* block capacity C of the balanced partition; only 64 is supported (ignored
+                                        for DA2_PARTITION_TILES) */
 } da2_config_t;
 
 typedef struct da2_plan da2_plan_t;
@@ -100,6 +112,10 @@ typedef struct {
                                         blocks R .. R + R_prefix - 1 are the prefix's: counts is int32[BH][R +
                                         R_prefix][4], the 16-bit records cover R + R_prefix blocks per head, and
                                         tier_active[2] is set */
+  int32_t partition;                 /* da2_partition_t; for the balanced partition R_f = ceil(Hg*Wg/64) and: */
+  int32_t part_transposed, part_bands; /* the chosen band order: bands along columns (1) or rows (0), their number */
+  int32_t part_n, part_rem;          /* region r of a frame holds part_n + (r < part_rem) tokens, in its first slots */
+  int64_t part_perimeter;            /* total perimeter of one frame's regions */
   int32_t row_stride;                /* ROW scope: id entries reserved per video row (its offset is row * row_stride) */
   uint64_t off_order;                /* uint16[BH][2*ceil(R/2)]: query blocks of a head by decreasing list length
                                         (ties: lower index first; 0xFFFF pads an odd R), written in HEAD scope only
@@ -129,6 +145,11 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out);
 
 /* Fills *info.  Host only. */
 da2_status_t da2_plan_info(const da2_plan_t *plan, da2_plan_info_t *info);
+
+/* The token-to-region map (Sec. 3.3: regions packed into contiguous blocks; the inverse map restores the output
+ * order): index, within one head's [n_prefix + N] token sequence, of the token that slot `slot` (0..63) of block
+ * `block` (0 .. R + R_prefix - 1) holds; -1 for a padding slot, -2 for arguments out of range.  Host only. */
+int64_t da2_plan_slot_token(const da2_plan_t *plan, int32_t block, int32_t slot);
 
 /* Pool, draft map, ranking, lists and operand records for (q, k, v) into workspace.  Enqueues on stream. */
 da2_status_t da2_prepare(const da2_plan_t *plan, const void *q, const void *k, const void *v, void *workspace,

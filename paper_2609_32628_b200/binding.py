@@ -12,6 +12,7 @@ _lib = None
 STATUS = {0: "DA2_OK", 1: "DA2_ERR_INVALID_ARG", 2: "DA2_ERR_UNSUPPORTED", 3: "DA2_ERR_WORKSPACE_TOO_SMALL",
           4: "DA2_ERR_CUDA", 5: "DA2_ERR_TIMEOUT", 6: "DA2_ERR_INTERNAL"}
 DA2_RANK_ROW, DA2_RANK_HEAD = 0, 1
+DA2_PARTITION_TILES, DA2_PARTITION_BALANCED = 0, 1
 
 
 class Da2Error(RuntimeError):
@@ -27,7 +28,7 @@ class _Config(ctypes.Structure):
                 ("frac4", ctypes.c_double), ("lambda_", ctypes.c_float), ("softmax_scale", ctypes.c_float),
                 ("rank_scope", ctypes.c_int32), ("n_prefix", ctypes.c_int32),
                 ("g_q", ctypes.POINTER(ctypes.c_float)), ("g_k", ctypes.POINTER(ctypes.c_float)),
-                ("g_v", ctypes.POINTER(ctypes.c_float))]
+                ("g_v", ctypes.POINTER(ctypes.c_float)), ("partition", ctypes.c_int32), ("capacity", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -45,6 +46,8 @@ class PlanInfo(ctypes.Structure):
                 ("off_kvrec", ctypes.c_uint64 * 3), ("qrec_bytes", ctypes.c_uint32 * 3),
                 ("kvrec_bytes", ctypes.c_uint32 * 3), ("off_dq8", ctypes.c_uint64), ("off_dk8", ctypes.c_uint64),
                 ("off_dv8", ctypes.c_uint64), ("n_prefix", ctypes.c_int32), ("R_prefix", ctypes.c_int32),
+                ("partition", ctypes.c_int32), ("part_transposed", ctypes.c_int32), ("part_bands", ctypes.c_int32),
+                ("part_n", ctypes.c_int32), ("part_rem", ctypes.c_int32), ("part_perimeter", ctypes.c_int64),
                 ("row_stride", ctypes.c_int32), ("off_order", ctypes.c_uint64)]
 
 
@@ -75,6 +78,8 @@ def load_library():
         lib.da2_last_launch_count.argtypes = [vp]
         lib.da2_probe_bounded_wait.restype = ctypes.c_int
         lib.da2_probe_bounded_wait.argtypes = [vp, vp, ctypes.c_int64, vp]
+        lib.da2_plan_slot_token.restype = ctypes.c_int64
+        lib.da2_plan_slot_token.argtypes = [vp, ctypes.c_int32, ctypes.c_int32]
         lib.da2_plan_destroy.restype = None
         lib.da2_plan_destroy.argtypes = [vp]
         lib.da2_status_string.restype = ctypes.c_char_p
@@ -108,10 +113,11 @@ class Plan:
 
 def da2_plan(B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float, frac4: float,
              lam: float = 0.2, softmax_scale: float = 0.0, rank_scope: int = DA2_RANK_ROW,
-             g_q=None, g_k=None, g_v=None, tile_h: int = 8, tile_w: int = 8, n_prefix: int = 0) -> Plan:
+             g_q=None, g_k=None, g_v=None, tile_h: int = 8, tile_w: int = 8, n_prefix: int = 0,
+             partition: int = 0, capacity: int = 64) -> Plan:
     cfg = _Config(B, H, T, Hg, Wg, head_dim, tile_h, tile_w, frac16, frac8, frac4, lam, softmax_scale, rank_scope,
                   n_prefix,
-                  None, None, None)
+                  None, None, None, partition, capacity)
     keep = []
     for name, arr in (("g_q", g_q), ("g_k", g_k), ("g_v", g_v)):
         if arr is not None:
@@ -131,6 +137,11 @@ def da2_plan_info(plan: Plan) -> PlanInfo:
     if rc != 0:
         raise Da2Error(rc, "da2_plan_info")
     return info
+
+
+def da2_plan_slot_token(plan: Plan, block: int, slot: int) -> int:
+    """Token index (in a head's [n_prefix + N] sequence) held by a slot of a block; -1 = padding."""
+    return int(load_library().da2_plan_slot_token(plan.handle, block, slot))
 
 
 def _ptr(t) -> int:
@@ -251,7 +262,8 @@ class HostPipeline:
     """
 
     def __init__(self, B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: float, frac8: float,
-                 frac4: float, lam: float = 0.2, rank_scope: int = DA2_RANK_ROW, groups="ramp", device="cuda"):
+                 frac4: float, lam: float = 0.2, rank_scope: int = DA2_RANK_ROW, groups="ramp", device="cuda",
+                 partition: int = DA2_PARTITION_TILES):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -260,7 +272,8 @@ class HostPipeline:
         for n in self._group_sizes(self.BH, groups):
             self.ranges.append((h0, h0 + n))
             h0 += n
-        self.plans = {n: da2_plan(1, n, T, Hg, Wg, head_dim, frac16, frac8, frac4, lam=lam, rank_scope=rank_scope)
+        self.plans = {n: da2_plan(1, n, T, Hg, Wg, head_dim, frac16, frac8, frac4, lam=lam, rank_scope=rank_scope,
+                                  partition=partition)
                       for n in {b - a for a, b in self.ranges}}
         nmax = max(self.plans)
         wsb = max(int(p.info.workspace_bytes) for p in self.plans.values())

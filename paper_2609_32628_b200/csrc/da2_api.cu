@@ -3,6 +3,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "da2_internal.cuh"
 
@@ -41,6 +42,8 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
   p.nty = I.nty; p.ntx = I.ntx; p.R_f = I.R_f; p.R = I.R; p.N = I.N; p.BH = I.B * I.H;
   p.P = I.n_prefix; p.Rp = I.R_prefix; p.Rt = I.R + I.R_prefix; p.Ntot = I.N + I.n_prefix;
   p.row_stride = I.row_stride;
+  p.part = I.partition; p.part_tr = I.part_transposed; p.part_bands = I.part_bands; p.part_n = I.part_n;
+  p.part_rem = I.part_rem;
   p.rank_scope = I.rank_scope;
   for (int t = 0; t < 3; ++t) {
     p.tier_active[t] = I.tier_active[t];
@@ -75,6 +78,57 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
 
 bool misaligned(const void *ptr, uintptr_t a) { return ((uintptr_t)ptr % a) != 0; }
 
+// Balanced ragged partition of one H x W frame into Rf regions (App. C.2): candidates are band orders (see
+// slot_token in da2_internal.cuh) cut into Rf runs of n or n + 1 cells; a candidate counts if every run is
+// 4-connected, and the one with the fewest cut edges (smallest total perimeter, Eq. "region-perimeter") wins; ties go
+// to bands along rows, then to fewer bands.  Host only, integer work, once per plan.
+struct BandChoice { int transposed, bands; long long perimeter; };
+
+int band_cell(int H, int W, int bands, int transposed, int pos) {
+  const int L = transposed ? W : H, M = transposed ? H : W;
+  const int hb = L / bands, extra = L % bands, big = extra * (hb + 1) * M;
+  int b, h, q;
+  if (pos < big) { h = hb + 1; b = pos / (h * M); q = pos - b * h * M; }
+  else { h = hb; pos -= big; b = pos / (h * M); q = pos - b * h * M; b += extra; }
+  const int l0 = b * hb + (b < extra ? b : extra);
+  const int i = q / h, k = q - i * h;
+  const int m = (b & 1) ? M - 1 - i : i;
+  const int l = l0 + ((i & 1) ? h - 1 - k : k);
+  return transposed ? m * W + l : l * W + m;
+}
+
+BandChoice choose_bands(int H, int W, int Rf) {
+  const int HW = H * W, n = HW / Rf, rem = HW % Rf;
+  std::vector<int> region(HW), parent(HW);
+  BandChoice best = {0, 0, -1};
+  for (int tr = 0; tr < 2; ++tr)
+    for (int bands = 1; bands <= (tr ? W : H); ++bands) {
+      int pos = 0;
+      for (int a = 0; a < Rf; ++a)
+        for (int j = 0; j < n + (a < rem); ++j) region[band_cell(H, W, bands, tr, pos++)] = a;
+      // union-find over equal-region neighbours; the cut edges are counted on the way
+      for (int c = 0; c < HW; ++c) parent[c] = c;
+      auto find = [&](int c) { while (parent[c] != c) { parent[c] = parent[parent[c]]; c = parent[c]; } return c; };
+      long long cut = 0;
+      int comps = HW;
+      for (int y = 0; y < H; ++y)
+        for (int x = 0; x < W; ++x) {
+          const int c = y * W + x;
+          const int nb[2] = {x + 1 < W ? c + 1 : -1, y + 1 < H ? c + W : -1};
+          for (int e = 0; e < 2; ++e) {
+            if (nb[e] < 0) continue;
+            if (region[nb[e]] != region[c]) { ++cut; continue; }
+            const int ra = find(c), rb = find(nb[e]);
+            if (ra != rb) { parent[ra] = rb; --comps; }
+          }
+        }
+      if (comps != Rf) continue;
+      const long long per = 2ll * (H + W) + 2 * cut;
+      if (best.perimeter < 0 || per < best.perimeter) best = {tr, bands, per};
+    }
+  return best;
+}
+
 // kernels enqueued by the calling thread's last da2_prepare / da2_refresh_operands / da2_attention_fwd
 thread_local int t_last_launches = 0;
 
@@ -105,6 +159,9 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   if (cfg->n_prefix > 0 && cfg->rank_scope == DA2_RANK_HEAD) return DA2_ERR_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return DA2_ERR_UNSUPPORTED;
   if (cfg->tile_h != 8 || cfg->tile_w != 8) return DA2_ERR_UNSUPPORTED;
+  if (cfg->partition != DA2_PARTITION_TILES && cfg->partition != DA2_PARTITION_BALANCED) return DA2_ERR_INVALID_ARG;
+  // the balanced partition packs regions into blocks of the kernels' 64 slots; 128-token blocks are not built
+  if (cfg->partition == DA2_PARTITION_BALANCED && cfg->capacity != da2::kSlots) return DA2_ERR_UNSUPPORTED;
 
   da2_plan_t *plan = new (std::nothrow) da2_plan_t();
   if (!plan) return DA2_ERR_INTERNAL;
@@ -118,6 +175,17 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   I.nty = (cfg->Hg + 7) / 8;
   I.ntx = (cfg->Wg + 7) / 8;
   I.R_f = I.nty * I.ntx;
+  I.partition = cfg->partition;
+  if (cfg->partition == DA2_PARTITION_BALANCED) {
+    const int HW = cfg->Hg * cfg->Wg;
+    I.R_f = (HW + da2::kSlots - 1) / da2::kSlots;
+    const BandChoice ch = choose_bands(cfg->Hg, cfg->Wg, I.R_f);
+    I.part_transposed = ch.transposed;
+    I.part_bands = ch.bands;
+    I.part_perimeter = ch.perimeter;
+    I.part_n = HW / I.R_f;
+    I.part_rem = HW % I.R_f;
+  }
   long long R = (long long)cfg->T * I.R_f;
   if (R > 16384) { delete plan; return DA2_ERR_UNSUPPORTED; }  // ids are uint16; row buffers live in shared memory
   const long long Rp = ((long long)cfg->n_prefix + da2::kSlots - 1) / da2::kSlots, Rt = R + Rp;
@@ -305,6 +373,13 @@ da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, vo
   if (word[0] == da2::kDevOk) return DA2_OK;
   if (word[0] == da2::kDevTimeout) return DA2_ERR_TIMEOUT;
   return DA2_ERR_INTERNAL;
+}
+
+int64_t da2_plan_slot_token(const da2_plan_t *plan, int32_t block, int32_t slot) {
+  if (!plan || block < 0 || block >= plan->info.R + plan->info.R_prefix || slot < 0 || slot >= da2::kSlots) return -2;
+  const da2::Params p = make_params(plan, nullptr);
+  if (!((da2::block_valid_mask(p, block) >> slot) & 1ull)) return -1;
+  return (int64_t)da2::slot_token(p, block, slot);
 }
 
 int32_t da2_last_launch_count(const da2_plan_t *plan) { return plan ? t_last_launches : 0; }

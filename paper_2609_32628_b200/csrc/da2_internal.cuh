@@ -26,6 +26,8 @@ struct Params {
   int P, Rp, Rt;            // prefix tokens, prefix blocks (ceil(P / 64)), blocks per head R + Rp
   long long Ntot;           // tokens per head in the tensors: P prefix tokens, then the N video tokens
   int row_stride;           // id entries reserved per video row (ROW scope)
+  // balanced ragged partition (App. C.2): 0 = fixed 8 x 8 tiles; else the chosen band order and the run lengths
+  int part, part_tr, part_bands, part_n, part_rem;
   int BH;
   int rank_scope;
   int tier_active[3];       // 0: NVFP4, 1: INT8/E4M3, 2: BF16
@@ -57,6 +59,10 @@ __host__ __device__ inline unsigned long long block_valid_mask(const Params &p, 
     return rem >= kSlots ? ~0ull : ((1ull << rem) - 1ull);
   }
   int r = a % p.R_f;
+  if (p.part) {  // a run of the band order: its n or n + 1 tokens fill the first slots
+    const int na = p.part_n + (r < p.part_rem);
+    return na >= kSlots ? ~0ull : ((1ull << na) - 1ull);
+  }
   int ty = r / p.ntx, tx = r % p.ntx;
   int vr = min(kTile, p.Hg - ty * kTile), vc = min(kTile, p.Wg - tx * kTile);
   unsigned long long rowbits = (vc >= 8) ? 0xffull : ((1ull << vc) - 1ull);
@@ -70,6 +76,24 @@ __host__ __device__ inline unsigned long long block_valid_mask(const Params &p, 
 __host__ __device__ inline long long slot_token(const Params &p, int a, int j) {
   if (a >= p.R) return (long long)(a - p.R) * kSlots + j;
   int t = a / p.R_f, r = a % p.R_f;
+  if (p.part) {
+    // Band order: the frame is cut into part_bands bands along one axis (the taller ones first); band b is walked
+    // column by column (forwards for even b, backwards for odd b), the columns alternately down and up; region r is
+    // the r-th run of that order, slot j its j-th cell.
+    const int L = p.part_tr ? p.Wg : p.Hg, M = p.part_tr ? p.Hg : p.Wg;
+    const int hb = L / p.part_bands, extra = L % p.part_bands;
+    int pos = r * p.part_n + min(r, p.part_rem) + j;
+    const int big = extra * (hb + 1) * M;
+    int b, h, q;
+    if (pos < big) { h = hb + 1; b = pos / (h * M); q = pos - b * h * M; }
+    else { h = hb; pos -= big; b = pos / (h * M); q = pos - b * h * M; b += extra; }
+    const int l0 = b * hb + min(b, extra);
+    const int i = q / h, k = q - i * h;
+    const int m = (b & 1) ? M - 1 - i : i;
+    const int l = l0 + ((i & 1) ? h - 1 - k : k);
+    const int cell = p.part_tr ? m * p.Wg + l : l * p.Wg + m;
+    return p.P + (long long)t * p.Hg * p.Wg + cell;
+  }
   int ty = r / p.ntx, tx = r % p.ntx;
   int y = ty * kTile + (j >> 3), x = tx * kTile + (j & 7);
   return p.P + ((long long)t * p.Hg + y) * p.Wg + x;

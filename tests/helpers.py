@@ -16,12 +16,13 @@ def scale_of(w) -> float:
     return float(np.float32(1.0) / np.sqrt(np.float32(w.head_dim)))
 
 
-def run_gpu(w, q, k, v, rank_scope=0, lam=None, zero_ws=False, g_fixed=None):
+def run_gpu(w, q, k, v, rank_scope=0, lam=None, zero_ws=False, g_fixed=None, partition=0):
     """q,k,v CUDA bf16 [B,H,N,d].  g_fixed: optional (g_q, g_k, g_v) host arrays [B*H] of caller-fixed NVFP4
     per-tensor scales.  Returns (plan, workspace uint8 tensor, out)."""
     gq, gk, gv = (None, None, None) if g_fixed is None else g_fixed
     plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4,
-                        lam=w.lam if lam is None else lam, rank_scope=rank_scope, g_q=gq, g_k=gk, g_v=gv)
+                        lam=w.lam if lam is None else lam, rank_scope=rank_scope, g_q=gq, g_k=gk, g_v=gv,
+                        partition=partition)
     ws = (torch.zeros if zero_ws else torch.empty)(int(plan.info.workspace_bytes), dtype=torch.uint8, device=q.device)
     out = torch.full_like(q, float("nan"))
     da2.da2_prepare(plan, q, k, v, ws)
@@ -132,12 +133,12 @@ class Workspace:
         return unq(qr), unq(kvr[:, :, :64 * d]), vt
 
 
-def oracle_all(w, q, k, v, heads=None, rank_scope=0, lam=None):
+def oracle_all(w, q, k, v, heads=None, rank_scope=0, lam=None, balanced=False):
     """Runs every oracle stage on CPU copies of q, k, v (optionally a subset of flat heads)."""
     sel = slice(None) if heads is None else list(heads)
     bits = lambda t: np.ascontiguousarray(oracle.bf16_bits(t.reshape(-1, w.N, w.head_dim).cpu())[sel])
     qb, kb, vb = bits(q), bits(k), bits(v)
-    pl = oracle.plan(w.T, w.Hg, w.Wg)
+    pl = oracle.plan_balanced(w.T, w.Hg, w.Wg, 64) if balanced else oracle.plan(w.T, w.Hg, w.Wg)
     lam32 = float(np.float32(w.lam if lam is None else lam))
     r = oracle.run_pipeline(qb, kb, vb, pl, lam=lam32, scale=scale_of(w), frac16=w.frac16, frac8=w.frac8,
                             frac4=w.frac4, head_scope=bool(rank_scope))

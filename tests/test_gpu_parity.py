@@ -113,7 +113,15 @@ def _check_attention(w, out, ref, sel, bad_rows, heads=None, g_fixed=None, dv_fi
     err_d = rel_l2(got, dense)
     print(f"[{w.name}] attention vs oracle: rel L2 {err:.3e}, max abs {mx:.3e}; vs dense fp64: rel L2 {err_d:.3e} "
           f"(oracle vs dense {rel_l2(exp, dense):.3e}) on {len(sel)} query blocks")
-    assert err <= 1e-2 and mx <= 2e-2
+    # bars: rel. L2 <= 1e-2 and max abs <= 2e-2.  The output is bf16: where |O| >= 4 its spacing (2^-5 and up) is
+    # wider than 2e-2, so a value whose exact result lies next to a rounding boundary can only differ by one unit
+    # in the last place or not at all; there the bar is that one unit (counted and printed).
+    diff = np.abs(got - exp)
+    ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(exp), 1e-30))) - 7)
+    wide = (np.abs(exp) >= 4.0) & (diff > 2e-2)
+    if wide.any():
+        print(f"[{w.name}] {int(wide.sum())} outputs with |O| >= 4 differ by one bf16 unit in the last place")
+    assert err <= 1e-2 and (diff <= np.where(np.abs(exp) >= 4.0, np.maximum(ulp, 2e-2), 2e-2)).all()
     return err, mx
 
 
@@ -202,21 +210,21 @@ def test_argument_errors_are_reported_before_any_launch():
     assert e.value.code == 1
 
 
-def _sampled_parity(name, nheads=2, nblocks=16, rank_scope=0, g_fixed=None):
+def _sampled_parity(name, nheads=2, nblocks=16, rank_scope=0, g_fixed=None, partition=0):
     """Full-size workload in the launch configuration the benchmark times; the oracle follows on sampled heads
     (every stage before attention in full for those heads) and on sampled query blocks for the attention output.
     The sample always holds the first and the last head (the last head's records lie beyond 2^31 bytes in the
     larger workspaces), both query blocks of two CTA pairs, one block of every edge-tile class and the last block."""
     w = da2_inputs.WORKLOADS[name]
     q, k, v = _inputs(w)
-    plan, ws, out = run_gpu(w, q, k, v, rank_scope=rank_scope, g_fixed=g_fixed)
+    plan, ws, out = run_gpu(w, q, k, v, rank_scope=rank_scope, g_fixed=g_fixed, partition=partition)
     BH, R = w.B * w.H, plan.info.R
     rng = np.random.default_rng(w.seed)
     heads = {0, BH - 1}
     while len(heads) < min(nheads, BH):
         heads.add(int(rng.integers(BH)))
     heads = sorted(heads)[:max(nheads, 1)] if nheads < 2 else sorted(heads)
-    ref = oracle_all(w, q, k, v, heads=heads, rank_scope=rank_scope)
+    ref = oracle_all(w, q, k, v, heads=heads, rank_scope=rank_scope, balanced=bool(partition))
     bad = _check_prepare(w, plan, ws, ref, heads=heads, g_fixed=g_fixed)
     R_f, ntx = plan.info.R_f, plan.info.ntx
     pair0, pair1 = 2 * int(rng.integers(R // 2)), 2 * int(rng.integers(R // 2))
@@ -235,6 +243,30 @@ def test_wan1p3b_480p_head_scope_sampled_parity():
     """Alg. 1 as printed (one ranking over all R*R pairs of a head) at a full-size configuration: rows of very
     different lengths, the scheduling order, CSR-style list offsets."""
     _sampled_parity("wan1p3b_480p", nheads=2, nblocks=16, rank_scope=1)
+
+
+@pytest.mark.parametrize("name", ["ragged3", "ragged64", "batch2"])
+@pytest.mark.parametrize("rank_scope", [0, 1])
+def test_balanced_partition_full_parity(name, rank_scope):
+    """The balanced ragged partition of App. C.2 (capacity 64) instead of fixed tiles: fewer blocks (12 x 20: 4
+    instead of 6 per frame; 9 x 13: 2 instead of 4), regions of 58 to 64 tokens packed into the first slots of their
+    blocks; every stage against the oracle on its own balanced plan, in both ranking scopes."""
+    w = SMALL[name]
+    q, k, v = _inputs(w)
+    plan, ws, out = run_gpu(w, q, k, v, rank_scope=rank_scope, partition=1)
+    ref = oracle_all(w, q, k, v, rank_scope=rank_scope, balanced=True)
+    assert plan.info.R == ref["pl"].R < oracle.plan(w.T, w.Hg, w.Wg).R or name == "batch2"
+    bad = _check_prepare(w, plan, ws, ref)
+    sel = [(h, a) for h in range(w.B * w.H) for a in range(plan.info.R)]
+    _check_attention(w, out, ref, sel, bad)
+    assert torch.isfinite(out.float()).all()
+
+
+@pytest.mark.parametrize("name", ["wan1p3b_480p", "wan14b_720p"])
+def test_balanced_partition_sampled_parity(name):
+    """Full-size configurations on the balanced partition: 25 instead of 28 blocks per 30 x 52 frame, 57 instead of 60
+    per 45 x 80 frame."""
+    _sampled_parity(name, nheads=2, nblocks=16, partition=1)
 
 
 def test_hunyuan_720p_sampled_parity():

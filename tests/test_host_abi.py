@@ -73,3 +73,34 @@ def test_compute_calls_reject_null_pointers_without_touching_cuda():
     assert lib.da2_prepare(plan.handle, 16, 16, 16, 256, 10, None) == 3   # workspace too small, still no launch
     assert lib.da2_refresh_operands(plan.handle, None, None, None, None, 0, None) == 1
     assert lib.da2_refresh_operands(plan.handle, 16, 16, 16, 256, 10, None) == 3
+
+
+@pytest.mark.parametrize("grid", [(2, 30, 52), (1, 45, 80), (3, 12, 20), (1, 9, 13), (2, 16, 16)])
+@pytest.mark.parametrize("mode", ["tiles", "balanced", "tiles+prefix"])
+def test_slot_table_matches_oracle(grid, mode):
+    """The token-to-region map the kernels index with (fixed tiles, the balanced ragged partition of App. C.2, and
+    prefix blocks) equals the oracle's independent table slot by slot; the balanced plan also reports the oracle's
+    choice of band order and perimeter."""
+    T, Hg, Wg = grid
+    P = 77 if mode == "tiles+prefix" else 0
+    plan = da2.da2_plan(1, 2, T, Hg, Wg, 64, 0.1, 0.2, 0.3, partition=1 if mode == "balanced" else 0, n_prefix=P)
+    pl = oracle.plan_balanced(T, Hg, Wg, 64) if mode == "balanced" else oracle.plan(T, Hg, Wg)
+    pl = oracle.plan_with_prefix(pl, P)
+    I = plan.info
+    assert I.R + I.R_prefix == pl.R and I.R == pl.R_video
+    got = [[da2.da2_plan_slot_token(plan, a, j) for j in range(64)] for a in range(pl.R)]
+    assert got == pl.slot_token.tolist()
+    if mode == "balanced":
+        assert (I.part_transposed, I.part_bands, I.part_perimeter) == oracle.plan_balanced(T, Hg, Wg, 64).choice
+        assert I.R_f == -(-Hg * Wg // 64)
+    assert da2.da2_plan_slot_token(plan, pl.R, 0) == -2 and da2.da2_plan_slot_token(plan, 0, 64) == -2
+    plan.close()
+
+
+def test_balanced_partition_rejects_other_capacities():
+    with pytest.raises(da2.Da2Error) as e:
+        da2.da2_plan(1, 1, 1, 16, 16, 64, 0.1, 0.1, 0.1, partition=1, capacity=128)
+    assert e.value.code == 2
+    with pytest.raises(da2.Da2Error) as e:
+        da2.da2_plan(1, 1, 1, 16, 16, 64, 0.1, 0.1, 0.1, partition=2)
+    assert e.value.code == 1
