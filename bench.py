@@ -328,6 +328,19 @@ def run_da2(args, rank, world, local_rank):
     e2e_ms = timed(lambda: pipe.run(hq, hk, hv, hout))
     assert pipe.status() == 0, "device status after the end-to-end region"
     e2e_launches = pipe.launches
+    del pipe
+    torch.cuda.empty_cache()
+    # the same pipeline inside the C ABI (da2_attention_host: synchronous, so timed on the host clock)
+    cfg = da2.make_config(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam,
+                          rank_scope=args.rank_scope, partition=args.partition)
+    arena = torch.empty(da2.da2_attention_host_arena_bytes(cfg), dtype=torch.uint8, device=dev)
+    da2.da2_attention_host(cfg, hq, hk, hv, hout, arena)
+    barrier()
+    tc0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        da2.da2_attention_host(cfg, hq, hk, hv, hout, arena)
+    e2e_c_ms = max_over_ranks((time.perf_counter() - tc0) * 1e3 / e2e_steps, world, dev)
+    del arena
     if rank != 0:
         return None
 
@@ -379,6 +392,7 @@ def run_da2(args, rank, world, local_rank):
                 "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": out.numel() * 2,
                 "how": f"HostPipeline: groups of {groups} heads, copy-in / kernels / copy-out on three streams, "
                        f"{e2e_launches} kernels per step",
+                "c_abi_host_entry_ms_per_step": e2e_c_ms,
                 "serial_ms_per_step": e2e_serial_ms,
                 "serial_value": dense * world / (e2e_serial_ms * 1e-3) / 1e12},
         "gpu_launches": launches, "clocks": clocks, "roofline": roofline,

@@ -186,6 +186,19 @@ da2_status_t da2_prepare_cached_scales(const da2_plan_t *plan, const void *q, co
 da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void *k, const void *v,
                                const void *workspace, void *out, void *stream);
 
+/* The whole call on HOST tensors (the paper has no counterpart: packaging).  hq, hk, hv, hout: HOST pointers, bf16
+ * [B, H, n_prefix + N, head_dim], ideally pinned (page-locked) so that the copies run asynchronously; arena: DEVICE
+ * memory, 256-byte aligned, at least da2_attention_host_arena_bytes() long, owned by the caller (the library
+ * allocates no device memory; it creates three streams and a few events for the duration of the call).  Heads are
+ * independent, so the call is cut into groups of heads (n_groups > 0: that many nearly equal groups; 0: small groups at
+ * both ends, large ones in between) whose host-to-device copies, kernels and device-to-host copies overlap on two
+ * device slots.  Synchronous: returns after the last copy; the return value includes the device status of every
+ * group (DA2_ERR_TIMEOUT / DA2_ERR_INTERNAL).  Caller-fixed g_q/g_k/g_v are not supported here
+ * (DA2_ERR_UNSUPPORTED).  The result is bit-identical to da2_prepare + da2_attention_fwd on the whole tensors. */
+da2_status_t da2_attention_host_arena_bytes(const da2_config_t *cfg, int32_t n_groups, size_t *bytes_out);
+da2_status_t da2_attention_host(const da2_config_t *cfg, const void *hq, const void *hk, const void *hv, void *hout,
+                                void *arena, size_t arena_bytes, int32_t n_groups);
+
 /* Synchronises stream, reads the workspace status word; DA2_OK, DA2_ERR_TIMEOUT or DA2_ERR_INTERNAL. */
 da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, void *stream);
 

@@ -131,6 +131,38 @@ def da2_plan(B: int, H: int, T: int, Hg: int, Wg: int, head_dim: int, frac16: fl
     return Plan(out.value)
 
 
+def _config(B, H, T, Hg, Wg, head_dim, frac16, frac8, frac4, lam=0.2, softmax_scale=0.0, rank_scope=DA2_RANK_ROW,
+            tile_h=8, tile_w=8, n_prefix=0, partition=0, capacity=64) -> _Config:
+    return _Config(B, H, T, Hg, Wg, head_dim, tile_h, tile_w, frac16, frac8, frac4, lam, softmax_scale, rank_scope,
+                   n_prefix, None, None, None, partition, capacity)
+
+
+make_config = _config
+
+
+def da2_attention_host_arena_bytes(cfg: _Config, n_groups: int = 0) -> int:
+    out = ctypes.c_size_t()
+    fn = load_library().da2_attention_host_arena_bytes
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.POINTER(_Config), ctypes.c_int32, ctypes.POINTER(ctypes.c_size_t)]
+    rc = fn(ctypes.byref(cfg), n_groups, ctypes.byref(out))
+    if rc != 0:
+        raise Da2Error(rc, "da2_attention_host_arena_bytes")
+    return int(out.value)
+
+
+def da2_attention_host(cfg: _Config, hq, hk, hv, hout, arena, n_groups: int = 0) -> None:
+    """Whole call on (pinned) HOST tensors through the C ABI's pipelined entry point; arena: CUDA uint8 tensor."""
+    fn = load_library().da2_attention_host
+    fn.restype = ctypes.c_int
+    vp = ctypes.c_void_p
+    fn.argtypes = [ctypes.POINTER(_Config), vp, vp, vp, vp, vp, ctypes.c_size_t, ctypes.c_int32]
+    rc = fn(ctypes.byref(cfg), hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hout.data_ptr(), _ptr(arena),
+            arena.numel() * arena.element_size(), n_groups)
+    if rc != 0:
+        raise Da2Error(rc, "da2_attention_host")
+
+
 def da2_plan_info(plan: Plan) -> PlanInfo:
     info = PlanInfo()
     rc = load_library().da2_plan_info(plan.handle, ctypes.byref(info))

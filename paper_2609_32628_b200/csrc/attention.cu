@@ -585,11 +585,18 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       }
       tc::fence_before_sync();
       warp_arrive(bar(s, B_SFREE + g));
-      if ((kmask.x & kmask.y) != 0xffffffffu) {  // ragged edge tile: padding keys take no part
+      if ((kmask.x & kmask.y) != 0xffffffffu) {  // padding keys take no part
+        if (kmask.x == 0xffffffffu && kmask.y == 0x7fffffffu) {
+          v[63] = -INFINITY;  // a region of 63 tokens (the balanced partition's common case): one padding slot
+        } else if (kmask.x == 0xffffffffu) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          v[c] = ((kmask.x >> c) & 1u) ? v[c] : -INFINITY;
-          v[32 + c] = ((kmask.y >> c) & 1u) ? v[32 + c] : -INFINITY;
+          for (int c = 0; c < 32; ++c) v[32 + c] = ((kmask.y >> c) & 1u) ? v[32 + c] : -INFINITY;
+        } else {  // ragged edge tile
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            v[c] = ((kmask.x >> c) & 1u) ? v[c] : -INFINITY;
+            v[32 + c] = ((kmask.y >> c) & 1u) ? v[32 + c] : -INFINITY;
+          }
         }
       }
       // maxima of the four 16-key groups (pairwise trees), then of the row

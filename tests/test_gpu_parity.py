@@ -446,6 +446,36 @@ def test_host_pipeline_equals_the_direct_call():
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), groups
 
 
+def test_c_abi_host_entry_equals_the_direct_call():
+    """da2_attention_host (the C ABI's own pipelined host-buffer path) gives the bits of one direct call, for the
+    default group ramp and for fixed group counts, also with a prefix and the balanced partition."""
+    for kw in (dict(), dict(n_prefix=70, partition=1)):
+        w = W("hostc", 1, 5, 64, 2, 16, 24, 0.1, 0.2, 0.3, seed=33)
+        P = kw.get("n_prefix", 0)
+        q, k, v = _inputs(w)
+        if P:
+            g = torch.Generator(device="cpu").manual_seed(7)
+            q, k, v = (torch.cat([torch.randn(w.B, w.H, P, w.head_dim, generator=g).to(torch.bfloat16).cuda(), x], 2)
+                       .contiguous() for x in (q, k, v))
+        plan = da2.da2_plan(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam, **kw)
+        ws = torch.empty(int(plan.info.workspace_bytes), dtype=torch.uint8, device="cuda")
+        out = torch.full_like(q, float("nan"))
+        da2.da2_prepare(plan, q, k, v, ws)
+        da2.da2_attention_fwd(plan, q, k, v, ws, out)
+        torch.cuda.synchronize()
+        hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
+        cfg = da2.make_config(w.B, w.H, w.T, w.Hg, w.Wg, w.head_dim, w.frac16, w.frac8, w.frac4, lam=w.lam, **kw)
+        for groups in (0, 1, 3):
+            arena = torch.empty(da2.da2_attention_host_arena_bytes(cfg, groups), dtype=torch.uint8, device="cuda")
+            hout = torch.full_like(hq, float("nan")).pin_memory()
+            da2.da2_attention_host(cfg, hq, hk, hv, hout, arena, groups)
+            assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), (kw, groups)
+        small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+        with pytest.raises(da2.Da2Error) as e:
+            da2.da2_attention_host(cfg, hq, hk, hv, hout, small, 0)
+        assert e.value.code == 3
+
+
 def test_scheduling_order_sorts_rows_by_list_length(rank_scope=1):
     """The order region pairs query blocks of equal list length: a permutation of the blocks of each head, by
     decreasing length, lower index first among equals, padded with 0xFFFF when R is odd."""
