@@ -36,54 +36,6 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
   return __half2float(*reinterpret_cast<const __half *>(&h));
 }
 
-__device__ __forceinline__ uint32_t cast_e4m3x2(float lo, float hi) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %2, %1;" : "=h"(r) : "f"(lo), "f"(hi));
-  return (uint32_t)r;
-}
-
-// Quantisation without a division per element, bit-identical to the definition code = cast(fl(x / s)).
-// With r = fl(1 / s) the product q = fl(x * r) is within a factor 1 +- 3 * 2^-24 of the correctly rounded quotient.
-// Every cast used here (round to nearest integer, E4M3, E2M1; saturating) is monotone, so when the two ends
-// q * (1 - 2^-21) and q * (1 + 2^-21) cast to the same code, the quotient, which lies strictly between them, casts to
-// that code as well.  Otherwise the product sits next to a rounding boundary (about one element in 10^5) and the
-// correctly rounded division decides.  Codes therefore stay reproducible bit for bit while the common path costs
-// three multiplications instead of a division.
-constexpr float kBelow = 1.0f - 0x1p-21f, kAbove = 1.0f + 0x1p-21f;
-// reciprocal of a scale; a scale so small that its reciprocal overflows has none, and every element then takes the
-// division (0 * inf would not compare)
-__device__ __forceinline__ float safe_rcp(float s) {
-  const float r = __frcp_rn(s);
-  return r < 3.0e38f ? r : -1.0f;  // negative marks "no reciprocal"
-}
-
-// INT8 code (round half away from zero, App. C.3).  Between two equal nearest-integer roundings no half-integer lies,
-// so the two rounding modes agree there.
-__device__ __forceinline__ int int8_code(float x, float delta, float rinv) {
-  const float q = __fmul_rn(x, rinv);
-  const int a = __float2int_rn(__fmul_rn(q, kBelow)), b = __float2int_rn(__fmul_rn(q, kAbove));
-  if (a == b && rinv > 0.f) return a;
-  return (int)roundf(__fdiv_rn(x, delta));
-}
-
-// two E4M3 codes (bits 7:0 and 15:8) of x / s
-__device__ __forceinline__ uint32_t e4m3x2_code(float x0, float x1, float s, float rinv) {
-  const float q0 = __fmul_rn(x0, rinv), q1 = __fmul_rn(x1, rinv);
-  const uint32_t a = cast_e4m3x2(__fmul_rn(q0, kBelow), __fmul_rn(q1, kBelow));
-  const uint32_t b = cast_e4m3x2(__fmul_rn(q0, kAbove), __fmul_rn(q1, kAbove));
-  if (a == b && rinv > 0.f) return a;
-  return cast_e4m3(__fdiv_rn(x0, s)) | (cast_e4m3(__fdiv_rn(x1, s)) << 8);
-}
-
-// two E2M1 codes (bits 3:0 and 7:4) of x / s
-__device__ __forceinline__ uint32_t e2m1x2_code(float x0, float x1, float s, float rinv) {
-  const float q0 = __fmul_rn(x0, rinv), q1 = __fmul_rn(x1, rinv);
-  const uint32_t a = cast_e2m1x2(__fmul_rn(q0, kBelow), __fmul_rn(q1, kBelow));
-  const uint32_t b = cast_e2m1x2(__fmul_rn(q0, kAbove), __fmul_rn(q1, kAbove));
-  if (a == b && rinv > 0.f) return a;
-  return cast_e2m1x2(__fdiv_rn(x0, s), __fdiv_rn(x1, s));
-}
-
 // NVFP4 group of 16 values (Eq. "v2-nvfp4-quantization"): returns the E4M3 scale code, writes 8 bytes of codes
 __device__ __forceinline__ uint32_t nvfp4_group(const float (&x)[16], float g, uint32_t (&packed)[2]) {
   float gmax = 0.f;
@@ -93,10 +45,10 @@ __device__ __forceinline__ uint32_t nvfp4_group(const float (&x)[16], float g, u
   const float sigma = decode_e4m3(sc);
   packed[0] = 0; packed[1] = 0;
   if (sigma == 0.f) return sc;  // a group whose encoded scale is zero is encoded as zero
-  const float step = __fmul_rn(g, sigma), rinv = safe_rcp(step);
+  const float step = __fmul_rn(g, sigma);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const uint32_t b = e2m1x2_code(x[2 * i], x[2 * i + 1], step, rinv);
+    const uint32_t b = cast_e2m1x2(__fdiv_rn(x[2 * i], step), __fdiv_rn(x[2 * i + 1], step));
     packed[i >> 2] |= b << (8 * (i & 3));
   }
   return sc;
@@ -211,14 +163,13 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
     uint8_t *kr = p.kvrec[1] + blk * p.kvrec_bytes[1];
     uint8_t *vr = kr + kSlots * D;
     const float dq = s_delta[0], dk = s_delta[1];
-    const float rq = safe_rcp(dq), rk = safe_rcp(dk);
     for (int idx = tid; idx < kSlots * D / 16; idx += NT) {  // chunk (kc, r): channels kc*16.. of slot r
       const int kc = idx / kSlots, r = idx % kSlots;
       uint32_t wq[4] = {0, 0, 0, 0}, wk[4] = {0, 0, 0, 0};
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        const int cq = int8_code(bf16_to_f32(tq[r * D + kc * 16 + i]), dq, rq);
-        const int ck = int8_code(bf16_to_f32(tk[r * D + kc * 16 + i]), dk, rk);
+        const int cq = (int)roundf(__fdiv_rn(bf16_to_f32(tq[r * D + kc * 16 + i]), dq));
+        const int ck = (int)roundf(__fdiv_rn(bf16_to_f32(tk[r * D + kc * 16 + i]), dk));
         wq[i >> 2] |= (uint32_t)(cq & 0xff) << (8 * (i & 3));
         wk[i >> 2] |= (uint32_t)(ck & 0xff) << (8 * (i & 3));
       }
@@ -230,15 +181,11 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
       const float dv = p.dv8[(size_t)bh * D + c];
       uint32_t w[4] = {0, 0, 0, 0};
       if (dv > 0.f) {
-        const float rv = safe_rcp(dv);
-        const uint32_t m16 = (uint32_t)(mask >> (kc * 16)) & 0xffffu;
 #pragma unroll
-        for (int i = 0; i < 16; i += 2) {
+        for (int i = 0; i < 16; ++i) {
           const int slot = kc * 16 + i;
-          uint32_t code = e4m3x2_code(bf16_to_f32(tv[slot * D + c]), bf16_to_f32(tv[(slot + 1) * D + c]), dv, rv);
-          // padding slots hold zeros in the staged tile; their codes are defined as 0 whatever the sign of zero
-          if (!((m16 >> i) & 1u)) code &= 0xff00u;
-          if (!((m16 >> (i + 1)) & 1u)) code &= 0x00ffu;
+          uint32_t code = 0;
+          if ((mask >> slot) & 1ull) code = cast_e4m3(__fdiv_rn(bf16_to_f32(tv[slot * D + c]), dv));
           w[i >> 2] |= code << (8 * (i & 3));
         }
       }
