@@ -7,18 +7,26 @@
 // the accumulator only changes units (Eq. "precision-state-conversion"), and the output is normalised once.
 //
 // Mapping onto sm_100a
-//   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 576 threads in five roles:
-//     warps 0-7   softmax: stream = (warp%4)/2; warps w and w+4 own the same 32 query rows and take alternate steps,
-//                 one thread per 64-key row; they read S from TMEM, keep h and a partial l, and write P~ (and its
-//                 NVFP4 scale factors) to shared memory
-//     warps 8-11  correction + epilogue: rescale the accumulator columns of queries whose maximum moved, apply the
-//                 per-channel unit change at a segment boundary, and finally normalise, transpose and store
-//     warps 12,13 S = Q K^T issue, one warp per stream (tcgen05.mma, accumulators in TMEM), two steps ahead
-//     warps 14,15 O^T += V^T P~^T issue, one warp per stream.  The issuing warps' instruction counts are on the
-//                 critical path of every step: their loops are warp-uniform (one elected lane issues), operand
-//                 descriptors are built once and only offset inside the loop
-//     warps 16,17 loaders, one per stream: K and V^T (+ scale factor) records by 1-D bulk copies into two rings; a
-//                 warp-uniform loop in which lane l holds list entry 32*batch + l (address, mask, key scale)
+//   A CTA owns two neighbouring query blocks ("streams" 0 and 1) and 1024 threads (768 when shared memory only
+//   leaves room for two softmax sets) in six roles, with S = 4 (or 2) softmax sets:
+//     warps 0..4S-1   softmax, set k = warp/4 takes the steps i = k (mod S); inside a set stream = (warp%4)/2 and one
+//                     thread owns one full 64-key row.  A thread reads its S row from TMEM, takes the running maximum
+//                     of step i-1 from the thread of the previous set through a shared-memory word tagged with the
+//                     step, keeps a partial denominator, and writes P~ (and its NVFP4 scale factors) into its set's
+//                     operand image.  These warps hold most of the register file (setmaxnreg).
+//     next 8 warps    correction + epilogue, four per stream: rescale the accumulator columns of queries whose
+//                     maximum moved and apply the per-channel unit change at a segment boundary ON REQUEST of the
+//                     PV-issue warp (most steps move no maximum and request nothing), and finally combine the sets'
+//                     partial denominators, normalise, transpose and store
+//     next 2 warps    S = Q K^T issue, one warp per stream (tcgen05.mma, accumulators in TMEM), two steps ahead
+//     next 2 warps    O^T += V^T P~^T issue, one warp per stream; reads the step's "maximum moved" ballots and asks
+//                     for a correction only when one is set or the tier changes.  The issuing warps' instruction
+//                     counts are on the critical path of every step: their loops are warp-uniform (one elected lane
+//                     issues), operand descriptors are built once and only offset inside the loop
+//     last 4 warps    loaders: per stream one warp for K (and the Q records) and one for V^T, 1-D bulk copies into
+//                     rings of their own (a K block is needed as soon as a score buffer is free, a V block only after
+//                     the step's weights are written, so the V ring is the deeper one); lane l holds list entry
+//                     32*batch + l (address, mask, key scale)
 //   S   = Q K^T   : M = 128, N = 64 keys, K = d.  The block-scaled instruction only exists at M = 128, so stream 0's
 //                   queries sit in rows 0..63 and stream 1's in rows 64..127 (its operand descriptor starts 1 KB
 //                   early); the other 64 rows of each product are don't-care.  S is double buffered.
@@ -27,7 +35,7 @@
 //                   per-channel unit changes (eta*delta_c^V, g_V/2688) per-lane scalars.
 //   kinds         : kind::f16 (BF16); kind::i8 for QK^T + kind::f8f6f4 E4M3 x E4M3 for PV (App. C.1); and
 //                   kind::mxf4nvf4 with E4M3 scales per 16 elements (NVFP4), scale factors moved by tcgen05.cp.
-// The softmax sets the pace (one ex2 per score on a 16-lane/clk unit, and a chain of hand-offs per step): the row
+// The softmax sets the pace (per score: one ex2 on a 16-lane/clk unit plus the quantisation arithmetic): the row
 // maximum is taken on raw accumulator values, the scale and the maximum are folded into one FMA feeding ex2, int32
 // scores become floats through a magic-number add, the NVFP4 group scale is folded into the exponent so the scaled
 // weight needs no extra multiply, and the exponentiate phase runs over the whole row in batches (all arguments, all
@@ -35,6 +43,7 @@
 // the three are interleaved per pair.
 // Every wait on an mbarrier is bounded; a wait that gives up records device status "timeout", all roles leave their
 // loops and the CTA exits normally after releasing TMEM.
+#include <type_traits>
 #include <cuda_fp8.h>
 
 #include "da2_internal.cuh"
@@ -44,11 +53,18 @@ namespace da2 {
 
 namespace {
 
-constexpr int kSoftmaxWarps = 8, kCorrWarps = 4;
-constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;  // warps 12, 13: Q K^T issue for stream 0, 1
-constexpr int kPvWarp0 = kMmaWarp0 + 2;                // warps 14, 15: V^T P^T issue for stream 0, 1
-constexpr int kLoadWarp0 = kPvWarp0 + 2;               // warps 16, 17: loader for stream 0, 1
-constexpr int NT = (kLoadWarp0 + 2) * 32;              // 576
+// Softmax warp sets: set k takes the steps i = k (mod SETS), one thread per 64-key row, four warps (one per TMEM lane
+// quarter) per set.  Plans without a 16-bit tier run four sets; a 16-bit tier needs 8 KB per P image and 16 KB ring
+// stages, which leaves shared memory for two.
+constexpr int kMaxSets = 4;
+template <int SETS> struct Roles {
+  static constexpr int kSoftmaxWarps = 4 * SETS, kCorrWarps = 8;  // four correction warps per stream
+  static constexpr int kMmaWarp0 = kSoftmaxWarps + kCorrWarps;    // Q K^T issue for stream 0, 1
+  static constexpr int kPvWarp0 = kMmaWarp0 + 2;                  // V^T P^T issue for stream 0, 1
+  static constexpr int kLoadWarp0 = kPvWarp0 + 2;                 // K loaders for stream 0, 1, then V loaders
+  static constexpr int NT = (kLoadWarp0 + 4) * 32;                // 1024 (four sets) or 768 (two): whole warpgroups
+  static constexpr int kShift = SETS == 4 ? 2 : 1, kMask = SETS - 1;
+};
 constexpr uint32_t kTmemCols = 512;
 // TMEM column map
 __host__ __device__ constexpr uint32_t col_s(int s, int buf) { return (uint32_t)(s * 2 + buf) * 64u; }
@@ -66,29 +82,32 @@ constexpr float kOffsetP8 = 8.807f;      // base-2 exponent offset (about log2 4
 // barrier indices inside one stream's group
 // (a parity wait can only tell the latest completion from the one before, so every barrier is laid out such that no
 // waiter can fall two completions behind: buffers indexed by step parity get one barrier per buffer)
-enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 8, B_VFREE = 12, B_SREADY = 16, B_SFREE = 18, B_PREADY = 20, B_XREADY = 22,
-       B_PVDONE = 24, B_ELL = 26, B_Q = 27, B_COUNT = 28 };
-constexpr int kMaxStages = 4, kInfoRing = 8;
+enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 10, B_VFREE = 14, B_SREADY = 20, B_SFREE = 24, B_PREADY = 26, B_CORRGO = 30,
+       B_CORRDONE = 31, B_PVDONE = 34, B_ELL = 38, B_Q = 39, B_COUNT = 40 };
+constexpr int kMaxK = 4, kMaxV = 6, kInfoRing = 8;
 
 struct SmemMap {
   uint32_t q[2][3];   // Q record per stream and tier
-  uint32_t kst[2][kMaxStages];  // K ring per stream (K image + its scale atoms)
-  uint32_t vst[2][kMaxStages];  // V ring per stream (V^T image + its scale atom)
+  uint32_t kst[2][kMaxK];  // K ring per stream (K image + its scale atoms)
+  uint32_t vst[2][kMaxV];  // V ring per stream (V^T image + its scale atom)
   int nk, nv;                   // ring depths
   uint32_t kbytes[3], vbytes[3];
-  uint32_t p[2][2];   // P operand images per stream, double buffered (64 x 64 x <= 2 bytes)
-  uint32_t sfp[2][2]; // P scale atoms (512 B)
-  uint32_t factor;    // float [2 streams][2][64]
-  uint32_t xmax;      // float [2][2 parity][2 halves][64]
-  uint32_t ell;       // float [2][2 halves][64]
+  uint32_t p[2][kMaxSets];   // P operand images per stream, one per softmax set (64 x 64 x <= 2 bytes)
+  uint32_t sfp[2][kMaxSets]; // P scale atoms (512 B)
+  uint32_t factor;    // float [2 streams][sets][64]
+  uint32_t hx;        // {float h, int step} [2][sets][64]: running maximum after a step, handed from thread to thread
+  uint32_t href;      // float [2][sets][64]: reference of each set's partial denominator
+  uint32_t ell;       // float [2][sets][64]
   uint32_t info;      // per stream, ring of kInfoRing steps: {u64 mask, float dk8, pad}
   uint32_t bars;      // uint64 [2][B_COUNT]
   uint32_t kstage, vstage;  // bytes per ring stage
-  uint32_t chg;             // uint32 [2 streams][2][2]: ballots of the queries whose maximum moved this step
+  uint32_t pbytes;          // bytes of one P image (the kSets images of a stream are contiguous)
+  uint32_t chg;             // uint32 [2 streams][sets][2]: ballots of the queries whose maximum moved this step
   uint32_t total;
+  bool fits;                // the layout fits the 227 KB a block may use
 };
 
-__host__ SmemMap make_smem_map(const Params &p) {
+__host__ SmemMap make_smem_map(const Params &p, int kSets) {
   SmemMap m;
   uint32_t cur = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = cur; cur = (cur + bytes + 127u) / 128u * 128u; return o; };
@@ -106,30 +125,39 @@ __host__ SmemMap make_smem_map(const Params &p) {
   const uint32_t q_end = cur;
   const uint32_t pbytes = p.tier_active[2] ? 8192u : (p.tier_active[1] ? 4096u : 2048u);
   // ring depths: as deep as shared memory allows (the K ring also serves as the 16 KB output staging tile)
-  const uint32_t fixed = 4 * pbytes + 4 * 512 + 1024 + 256 + 2048 + 1024 + 2 * kInfoRing * 16 +
-                         2 * B_COUNT * 8 + 1024;
-  const uint32_t budget = 232448u - q_end - fixed;
-  const int cand[5][2] = {{4, 4}, {3, 4}, {3, 3}, {2, 3}, {2, 2}};
-  m.nk = 2; m.nv = 2;
-  for (int c = 0; c < 5; ++c) {
-    if (2u * (cand[c][0] * kstage + cand[c][1] * vstage) <= budget) { m.nk = cand[c][0]; m.nv = cand[c][1]; break; }
+  auto r128 = [](uint32_t b) { return (b + 127u) / 128u * 128u; };
+  const uint32_t fixed = 2 * kSets * (pbytes + 512) + 3 * r128(2 * kSets * 64 * 4) + r128(2 * kSets * 2 * 4) +
+                         r128(2 * kSets * 64 * 8) + r128(2 * kInfoRing * 16) + r128(2 * B_COUNT * 8);
+  const uint32_t budget = q_end + fixed < 232448u ? 232448u - q_end - fixed : 0u;
+  // a K block is consumed as soon as a score buffer is free (two per stream), a V block only after the weights of
+  // its step are written: the V ring is the deep one
+  const int cand[7][2] = {{3, 6}, {3, 5}, {3, 4}, {2, 4}, {2, 3}, {2, 2}, {2, 2}};
+  m.nk = 2; m.nv = 2; m.fits = false;
+  for (int c = 0; c < 7; ++c) {
+    if (2u * (cand[c][0] * kstage + cand[c][1] * vstage) <= budget) {
+      m.nk = cand[c][0]; m.nv = cand[c][1]; m.fits = true;
+      break;
+    }
   }
   while ((uint32_t)m.nk * kstage < 16384u) kstage += 128u;
   m.kstage = kstage; m.vstage = vstage;
   for (int s = 0; s < 2; ++s) {
-    for (int g = 0; g < kMaxStages; ++g) m.kst[s][g] = g < m.nk ? take(kstage) : 0;
+    for (int g = 0; g < kMaxK; ++g) m.kst[s][g] = g < m.nk ? take(kstage) : 0;
   }
   for (int s = 0; s < 2; ++s)
-    for (int g = 0; g < kMaxStages; ++g) m.vst[s][g] = g < m.nv ? take(vstage) : 0;
-  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.p[s][g] = take(pbytes);
-  for (int s = 0; s < 2; ++s) for (int g = 0; g < 2; ++g) m.sfp[s][g] = take(512);
-  m.factor = take(2 * 2 * 64 * 4);
-  m.chg = take(2 * 2 * 2 * 4);
-  m.xmax = take(2 * 2 * 2 * 64 * 4);
-  m.ell = take(2 * 2 * 64 * 4);
+    for (int g = 0; g < kMaxV; ++g) m.vst[s][g] = g < m.nv ? take(vstage) : 0;
+  m.pbytes = pbytes;
+  for (int s = 0; s < 2; ++s) for (int g = 0; g < kSets; ++g) m.p[s][g] = take(pbytes);
+  for (int s = 0; s < 2; ++s) for (int g = 0; g < kSets; ++g) m.sfp[s][g] = take(512);
+  m.factor = take(2 * kSets * 64 * 4);
+  m.chg = take(2 * kSets * 2 * 4);
+  m.hx = take(2 * kSets * 64 * 8);
+  m.href = take(2 * kSets * 64 * 4);
+  m.ell = take(2 * kSets * 64 * 4);
   m.info = take(2 * kInfoRing * 16);
   m.bars = take(2 * B_COUNT * 8);
   m.total = cur;
+  if (cur > 232448u) m.fits = false;
   return m;
 }
 
@@ -229,6 +257,16 @@ __device__ __forceinline__ void warp_arrive(uint64_t *bar) {
   if ((threadIdx.x & 31) == 0) tc::mbar_arrive(bar);
 }
 
+// register rebalancing between warpgroups: the softmax warps hold a whole score row, the others a few scalars
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+__device__ __forceinline__ uint2 ld_shared_volatile_v2(uint32_t saddr) {
+  uint2 r;
+  asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(saddr) : "memory");
+  return r;
+}
+
 struct StreamInfo {
   int a;         // query block, or -1
   int n4, n48;   // end of the NVFP4 segment, end of the INT8 segment (list positions)
@@ -254,11 +292,15 @@ __device__ __forceinline__ StreamInfo load_stream(const Params &p, int bh, int a
 // otherwise they are blocks 2p and 2p+1 (per-row budgets: every row has the same length, the order is the identity).
 // FP4: the plan has an NVFP4 tier.  Without one the exponentiate phase keeps the per-pair interleaved form, which is
 // the faster one for the 8-bit and bf16 bodies alone (the compiler's schedule of the unrolled softmax body decides).
-template <int D, bool ORDERED, bool FP4>
-__global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
+template <int D, bool ORDERED, bool FP4, int SETS>
+__global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p, SmemMap sm, __nv_bfloat16 *__restrict__ out) {
+  constexpr int kSets = SETS, NT = Roles<SETS>::NT, kSoftmaxWarps = Roles<SETS>::kSoftmaxWarps;
+  constexpr int kMmaWarp0 = Roles<SETS>::kMmaWarp0, kPvWarp0 = Roles<SETS>::kPvWarp0, kLoadWarp0 = Roles<SETS>::kLoadWarp0;
+  constexpr int kShift = Roles<SETS>::kShift, kMask = Roles<SETS>::kMask;
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
+  __shared__ int s_req[2];  // step a stream's correction warps are asked to rescale for
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
@@ -290,32 +332,37 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + sm.bars);
   auto bar = [&](int s, int which) -> uint64_t * { return bars + s * B_COUNT + which; };
-  float *s_factor = reinterpret_cast<float *>(smem + sm.factor);      // [s][buf][64]
-  uint32_t *s_chg = reinterpret_cast<uint32_t *>(smem + sm.chg);      // [s][buf][2]
-  float *s_xmax = reinterpret_cast<float *>(smem + sm.xmax);          // [s][parity][half][64]
-  float *s_ell = reinterpret_cast<float *>(smem + sm.ell);            // [s][half][64]
+  float *s_factor = reinterpret_cast<float *>(smem + sm.factor);      // [s][set][64]
+  uint32_t *s_chg = reinterpret_cast<uint32_t *>(smem + sm.chg);      // [s][set][2]
+  uint2 *s_hx = reinterpret_cast<uint2 *>(smem + sm.hx);              // [s][set][64]
+  float *s_href = reinterpret_cast<float *>(smem + sm.href);          // [s][set][64]
+  float *s_ell = reinterpret_cast<float *>(smem + sm.ell);            // [s][set][64]
   uint8_t *s_info = smem + sm.info;                                   // [s][kInfoRing] 16 bytes
 
+  for (int k_ = tid; k_ < 2 * kSets * 64; k_ += NT) s_hx[k_] = make_uint2(0u, 0xffffffffu);  // no step has this tag
   if (warp == 0) {
     tc::tmem_alloc(&s_tmem_base, kTmemCols);
     tc::tmem_relinquish();
   }
   if (tid == 32) {
     for (int s = 0; s < 2; ++s) {
-      for (int g = 0; g < 2; ++g) {
+      for (int g = 0; g < 2; ++g) tc::mbar_init(bar(s, B_SFREE + g), 2);
+      for (int g = 0; g < kSets; ++g) {
         tc::mbar_init(bar(s, B_SREADY + g), 1);
-        tc::mbar_init(bar(s, B_SFREE + g), 2);
-        tc::mbar_init(bar(s, B_PREADY + g), 6);  // 2 softmax warps (P written) + 4 correction warps (O rescaled)
-        tc::mbar_init(bar(s, B_XREADY + g), 2);
+        tc::mbar_init(bar(s, B_PREADY + g), 2);  // the two softmax warps of the step (P written)
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
       }
-      for (int g = 0; g < kMaxStages; ++g) {
+      for (int g = 0; g < kMaxK; ++g) {
         tc::mbar_init(bar(s, B_FULLK + g), 1);
-        tc::mbar_init(bar(s, B_FULLV + g), 1);
         tc::mbar_init(bar(s, B_KFREE + g), 1);
+      }
+      for (int g = 0; g < kMaxV; ++g) {
+        tc::mbar_init(bar(s, B_FULLV + g), 1);
         tc::mbar_init(bar(s, B_VFREE + g), 1);
       }
-      tc::mbar_init(bar(s, B_ELL), 4);
+      tc::mbar_init(bar(s, B_ELL), 2 * kSets);
+      tc::mbar_init(bar(s, B_CORRGO), 1);
+      tc::mbar_init(bar(s, B_CORRDONE), 4);
       tc::mbar_init(bar(s, B_Q), 1);
     }
     tc::fence_barrier_init();
@@ -327,210 +374,13 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
   const uint32_t tmem = s_tmem_base;
   volatile int *abortp = &s_abort;
 
-  // =========================================================================================== loader warps
-  if (warp >= kLoadWarp0) {
-    // Warp-uniform loop.  Lane l holds list entry 32 * batch + l ready for use: the record's address, the valid-key
-    // mask and the INT8 key scale; the ids of the next two batches and the scales of the next one are already on
-    // their way while a batch is used, so that a step costs a few shuffles and the copy requests of one elected lane.
-    const int s = warp - kLoadWarp0;
-    StreamInfo S = s ? st1 : st0;
-    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
-    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
-    S.L = __shfl_sync(0xffffffffu, S.L, 0);
-    if (S.L > 0) {
-      if (tc::elect_one()) {
-        const int nn[3] = {S.n4, S.n48 - S.n4, S.L - S.n48};
-        uint32_t bytes = 0;
-        for (int t = 0; t < 3; ++t) if (nn[t] > 0) bytes += p.qrec_bytes[t];
-        tc::mbar_arrive_expect_tx(bar(s, B_Q), bytes);
-        for (int t = 0; t < 3; ++t)
-          if (nn[t] > 0)
-            tc::bulk_g2s(smem + sm.q[s][t], p.qrec[t] + ((size_t)bh * rec_blocks(p, t) + S.a) * p.qrec_bytes[t], p.qrec_bytes[t],
-                         bar(s, B_Q));
-      }
-      __syncwarp();
-      const size_t head_blocks = (size_t)bh * R;
-      auto list_id = [&](int idx) -> int {
-        int b = idx < S.L ? (int)S.ids[idx] : 0;
-        if (b >= Rt) { atomicExch(p.status, kDevBadList); b = 0; }
-        return b;
-      };
-      auto key_scale = [&](int idx, int b) -> float {
-        return (idx < S.L && S.tier(idx) == 1) ? p.dk8[head_blocks + b] : 0.f;
-      };
-      auto record = [&](int idx, int b) -> unsigned long long {
-        const int t = S.tier(idx);
-        return reinterpret_cast<unsigned long long>(p.kvrec[t] + ((size_t)bh * rec_blocks(p, t) + b) * p.kvrec_bytes[t]);
-      };
-      int nxt_b = list_id(32 + lane), nn_b = list_id(64 + lane);
-      float cur_dk, nxt_dk = key_scale(32 + lane, nxt_b);
-      unsigned long long cur_rec, cur_mask;
-      {
-        const int b = list_id(lane);
-        cur_dk = key_scale(lane, b);
-        cur_rec = record(lane, b);
-        cur_mask = block_valid_mask(p, b);
-      }
-      const uint32_t kb0 = sm.kbytes[0], kb1 = sm.kbytes[1], kb2 = sm.kbytes[2];
-      const uint32_t vb0 = sm.vbytes[0], vb1 = sm.vbytes[1], vb2 = sm.vbytes[2];
-      uint8_t *kdst = smem + sm.kst[s][0], *vdst = smem + sm.vst[s][0];
-      int kk = 0, vv = 0;           // ring slots
-      uint32_t kpar = 1, vpar = 1;  // parity of the consumption that frees the slot (first pass: nothing to wait for)
-      bool kwrapped = false, vwrapped = false;
-      for (int i = 0; i < S.L; ++i) {
-        const int src = i & 31;
-        const uint32_t rlo = __shfl_sync(0xffffffffu, (uint32_t)cur_rec, src);
-        const uint32_t rhi = __shfl_sync(0xffffffffu, (uint32_t)(cur_rec >> 32), src);
-        const uint32_t mlo = __shfl_sync(0xffffffffu, (uint32_t)cur_mask, src);
-        const uint32_t mhi = __shfl_sync(0xffffffffu, (uint32_t)(cur_mask >> 32), src);
-        const float dk = __shfl_sync(0xffffffffu, cur_dk, src);
-        const uint8_t *rec = reinterpret_cast<const uint8_t *>(((unsigned long long)rhi << 32) | rlo);
-        const uint32_t kb = i < S.n4 ? kb0 : (i < S.n48 ? kb1 : kb2);
-        const uint32_t vb = i < S.n4 ? vb0 : (i < S.n48 ? vb1 : vb2);
-        if (kwrapped && !wait_or_abort(bar(s, B_KFREE + kk), kpar, abortp)) break;
-        if (tc::elect_one()) {
-          // the step's mask and key scale enter the info ring before the data the softmax waits for is requested
-          *reinterpret_cast<uint4 *>(s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16) =
-              make_uint4(mlo, mhi, __float_as_uint(dk), 0u);
-          tc::mbar_arrive_expect_tx(bar(s, B_FULLK + kk), kb);
-          tc::bulk_g2s(kdst + kk * sm.kstage, rec, kb, bar(s, B_FULLK + kk));
-        }
-        __syncwarp();
-        if (vwrapped && !wait_or_abort(bar(s, B_VFREE + vv), vpar, abortp)) break;
-        if (tc::elect_one()) {
-          tc::mbar_arrive_expect_tx(bar(s, B_FULLV + vv), vb);
-          tc::bulk_g2s(vdst + vv * sm.vstage, rec + kb, vb, bar(s, B_FULLV + vv));
-        }
-        __syncwarp();
-        if (++kk == sm.nk) { kk = 0; kpar ^= 1u; kwrapped = true; }
-        if (++vv == sm.nv) { vv = 0; vpar ^= 1u; vwrapped = true; }
-        if (src == 31) {  // next batch: its ids and scales were requested one batch ago
-          const int b = nxt_b;
-          cur_dk = nxt_dk;
-          cur_rec = record(i + 1 + lane, b);
-          cur_mask = block_valid_mask(p, b);
-          nxt_b = nn_b;
-          nxt_dk = key_scale(i + 33 + lane, nxt_b);
-          nn_b = list_id(i + 65 + lane);
-        }
-      }
-    }
-  }
-  // =========================================================================================== MMA warps
-  else if (warp >= kMmaWarp0 && warp < kPvWarp0) {
-    // The whole warp runs this loop with warp-uniform control flow and values; only the tcgen05 instructions
-    // themselves are issued by one elected lane.  (Under a lane-0 branch every descriptor would have to be moved from
-    // vector to uniform registers before each issue, which costs more than the MMA itself.)
-    const int s = warp - kMmaWarp0;
-    StreamInfo S = s ? st1 : st0;
-    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
-    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
-    S.L = __shfl_sync(0xffffffffu, S.L, 0);
-    if (S.L > 0 && wait_or_abort(bar(s, B_Q), 0, abortp)) {
-      // operand descriptors, built once; inside the loop only the 16-byte-unit start address (low bits) moves
-      const uint64_t qd0 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) - (s ? 1024u : 0u), 1024, 128);
-      const uint64_t qd1 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][1]) - (s ? 1024u : 0u), 1024, 128);
-      const uint64_t qd2 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][2]) - (s ? 1024u : 0u), 1024, 128);
-      const uint64_t kd0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]), 1024, 128);
-      const uint64_t ksf0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]) + kSlots * D / 2, 128, 128);
-      const uint32_t kstep = sm.kstage >> 4;
-      const uint32_t t_sfq = tmem + col_sfq(s), t_sfk = tmem + col_sfk(s);
-      if (S.n4 > 0) {  // Q scale factors go to TMEM once; the record carries them for rows 0..63 and again for rows
-                       // 64..127, so the same atom serves either stream
-        if (tc::elect_one()) {
-#pragma unroll
-          for (int k = 0; k < D / 64; ++k)
-            tc::tmem_cp_sf(t_sfq + 4 * k, tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) + kSlots * D / 2 + k * kSfAtomBytes,
-                                                         128, 128));
-        }
-      }
-      int kk = 0;
-      uint32_t kpar = 0;
-      // the score tiles are double buffered, so Q K^T runs up to two steps ahead of the softmax
-      for (int j = 0; j < S.L; ++j) {
-        const int g = j & 1;
-        if (!wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp)) break;
-        if (!wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp)) break;
-        tc::fence_after_sync();
-        const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
-        const uint32_t d_s = tmem + col_s(s, g);
-        if (tc::elect_one()) {
-          if (j >= S.n48) {
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
-          } else if (j >= S.n4) {
-#pragma unroll
-            for (int ks = 0; ks < D / 32; ++ks) tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
-          } else {
-            const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
-#pragma unroll
-            for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
-#pragma unroll
-            for (int ks = 0; ks < D / 64; ++ks)
-              tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks, t_sfk + 4 * ks);
-          }
-          tc::mma_commit(bar(s, B_SREADY + g));
-          tc::mma_commit(bar(s, B_KFREE + kk));
-        }
-        __syncwarp();
-        if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
-      }
-    }
-  }
-  // =========================================================================================== PV warps
-  else if (warp >= kPvWarp0) {
-    const int s = warp - kPvWarp0;
-    StreamInfo S = s ? st1 : st0;
-    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
-    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
-    S.L = __shfl_sync(0xffffffffu, S.L, 0);
-    if (S.L > 0) {
-      const uint64_t vd0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]), D * 16, 128);
-      const uint64_t vsf0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]) + D * kSlots / 2, 128, 128);
-      const uint64_t pd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.p[s][0]), 1024, 128),
-                              tc::smem_desc(tc::smem_u32(smem + sm.p[s][1]), 1024, 128)};
-      const uint64_t sfpd[2] = {tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][0]), 128, 128),
-                                tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][1]), 128, 128)};
-      const uint32_t vstep = sm.vstage >> 4;
-      const uint32_t t_sfv = tmem + col_sfv(s), t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
-      int vv = 0;
-      uint32_t vpar = 0;
-      for (int j = 0; j < S.L; ++j) {
-        // ---- O^T += V(j)^T P(j)^T, once P(j) is written and the accumulator is rescaled for step j
-        const int g = j & 1;
-        if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
-        if (!wait_or_abort(bar(s, B_PREADY + g), (j >> 1) & 1, abortp)) break;
-        tc::fence_after_sync();
-        const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
-        const uint32_t acc = j > 0;
-        if (tc::elect_one()) {
-          if (j >= S.n48) {
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              tc::mma_f16(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
-          } else if (j >= S.n4) {
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks)
-              tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pd[g] + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
-          } else {
-            tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
-            tc::tmem_cp_sf(t_sfp, sfpd[g]);
-            tc::mma_nvfp4(t_o, vd, pd[g], tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
-          }
-          tc::mma_commit(bar(s, B_PVDONE + g));
-          tc::mma_commit(bar(s, B_VFREE + vv));
-        }
-        __syncwarp();
-        if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
-      }
-    }
-  }
   // =========================================================================================== softmax warps
-  else if (warp < kSoftmaxWarps) {
-    // The two softmax warps that share a scheduler (warp w and w+4) own the same 32 query rows and take ALTERNATE
-    // steps, one thread per full 64-key row: while one exponentiates and packs its step (special-function bound),
-    // the other fetches, masks and reduces the next one.  The only hand-off between them is the running maximum.
-    const int s = (warp & 3) >> 1, par = warp >> 2;
+  if (warp < kSoftmaxWarps) {
+    reg_inc<(SETS == 4 ? 88 : 128)>();
+    // The warps w, w+4, w+8, ... share a scheduler and own the same 32 query rows; they take the steps of their sets
+    // in turn, one thread per full 64-key row: while one exponentiates and packs its step (special-function bound),
+    // the others fetch, mask and reduce later ones.  The only hand-off between them is the running maximum.
+    const int s = (warp & 3) >> 1, set = warp >> 2;
     const int r = (warp & 1) * 32 + lane;  // query row inside the stream's block
     const StreamInfo S = s ? st1 : st0;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -538,15 +388,15 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
     const float dq8s = (S.a >= 0 && S.a < R && p.tier_active[1]) ? p.dq8[(size_t)bh * R + S.a] * p.scale * kLog2e : 0.f;
     const float c16 = p.scale * kLog2e;
     float h_own = -INFINITY, ell = 0.f;  // log2-domain maximum after this warp's last step; its partial denominator
-    const int g = par;                   // buffers of this warp's step parity
-    float *my_h = s_xmax + ((s * 2 + g) * 2 + 0) * 64 + r;           // published running maximum of my steps
-    const float *other_h = s_xmax + ((s * 2 + (g ^ 1)) * 2 + 0) * 64 + r;
-    const uint32_t s_col = tmem + lane_addr + col_s(s, g);
+    const int g = set;                   // P buffer, barriers and hand-off slot of this set
+    uint2 *my_hx = s_hx + (s * kSets + set) * 64 + r;                // running maximum after my steps, tagged with the step
+    const uint32_t prev_hx = tc::smem_u32(s_hx + (s * kSets + ((set + kSets - 1) % kSets)) * 64 + r);
     uint8_t *prow = smem + sm.p[s][g] + r * 16;
 
-    for (int i = par; i < S.L; i += 2) {
+    for (int i = set; i < S.L; i += kSets) {
       const int tier = S.tier(i);
-      const uint32_t kp = (uint32_t)(i >> 1) & 1u;  // completion parity of this parity's k-th step
+      const uint32_t kp = (uint32_t)(i >> kShift) & 1u;  // completion parity of this set's k-th step
+      const uint32_t s_col = tmem + lane_addr + col_s(s, i & 1);
       if (!wait_or_abort(bar(s, B_SREADY + g), kp, abortp)) break;
       tc::fence_after_sync();
       // the step's mask and key scale (written before its K block was requested) are read while the scores load
@@ -584,7 +434,7 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
         }
       }
       tc::fence_before_sync();
-      warp_arrive(bar(s, B_SFREE + g));
+      warp_arrive(bar(s, B_SFREE + (i & 1)));
       if ((kmask.x & kmask.y) != 0xffffffffu) {  // padding keys take no part
         if (kmask.x == 0xffffffffu && kmask.y == 0x7fffffffu) {
           v[63] = -INFINITY;  // a region of 63 tokens (the balanced partition's common case): one padding slot
@@ -604,20 +454,29 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
 #pragma unroll
       for (int q = 0; q < 4; ++q) gm[q] = max16(v + q * 16);
       const float pmax = fmaxf(max3(gm[0], gm[1], gm[2]), gm[3]) * coef;  // log2 domain
-      // PV(i-2) done: this parity's P buffer is free and the correction warps are past step i-2
-      if (i >= 2 && !wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp)) break;
-      // running maximum after step i-1, published by the other warp
+      // PV(i-4) done: this set's P buffer is free and the correction warps are past step i-4
+      if (i >= kSets && !wait_or_abort(bar(s, B_PVDONE + g), (kp ^ 1u), abortp)) break;
+      // running maximum after step i-1: the thread that owns this row in the previous set leaves it, tagged with its
+      // step, in shared memory (one 8-byte store, one 8-byte load: no barrier on this chain)
       float h_prev = -INFINITY;
       if (i > 0) {
-        if (!wait_or_abort(bar(s, B_XREADY + (g ^ 1)), (uint32_t)((i - 1) >> 1) & 1u, abortp)) break;
-        h_prev = *other_h;
+        uint2 hv = ld_shared_volatile_v2(prev_hx);
+        for (uint32_t spin = 0; hv.y != (uint32_t)(i - 1); ++spin) {
+          if ((spin & 1023u) == 1023u && (*abortp || spin > (1u << 24))) break;
+          hv = ld_shared_volatile_v2(prev_hx);
+        }
+        const bool got = hv.y == (uint32_t)(i - 1);
+        if (!__all_sync(0xffffffffu, got)) {
+          atomicCAS(const_cast<int *>(abortp), 0, 1 + (int)(tc::smem_u32(bar(s, B_CORRGO)) & 0xffff));
+          break;
+        }
+        h_prev = __uint_as_float(hv.x);
       }
       const float m_new = fmaxf(h_prev, pmax);
-      *my_h = m_new;
-      s_factor[(s * 2 + g) * 64 + r] = ex2(h_prev - m_new);  // 0 on the first block (h_prev = -inf)
+      *my_hx = make_uint2(__float_as_uint(m_new), (uint32_t)i);
+      s_factor[(s * kSets + g) * 64 + r] = ex2(h_prev - m_new);  // 0 on the first block (h_prev = -inf)
       const uint32_t moved = __ballot_sync(0xffffffffu, m_new != h_prev);
-      if (lane == 0) s_chg[(s * 2 + g) * 2 + (warp & 1)] = moved;
-      warp_arrive(bar(s, B_XREADY + g));  // the other warp's next step and the correction warps wait on this
+      if (lane == 0) s_chg[(s * kSets + g) * 2 + (warp & 1)] = moved;
       ell *= ex2(h_own - m_new);
       h_own = m_new;
 
@@ -748,71 +607,284 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       warp_arrive(bar(s, B_PREADY + g));
     }
     if (S.L > 0) {
-      s_ell[(s * 2 + par) * 64 + r] = ell;
-      s_xmax[((s * 2 + par) * 2 + 1) * 64 + r] = h_own;  // reference of this partial denominator
+      s_ell[(s * kSets + set) * 64 + r] = ell;
+      s_href[(s * kSets + set) * 64 + r] = h_own;  // reference of this partial denominator
       warp_arrive(bar(s, B_ELL));
+    }
+  }
+  // =========================================================================================== loader warps
+  else {
+  reg_dec<40>();
+  if (warp >= kLoadWarp0) {
+    // Warps kLoadWarp0 + s request the K blocks of stream s (and its Q records), warps kLoadWarp0 + 2 + s its V
+    // blocks: a K block is consumed as soon as a score buffer is free, a V block only once the weights of its step
+    // are written, several steps later, so the two rings advance independently.
+    // Warp-uniform loop.  Lane l holds list entry 32 * batch + l ready for use: the record's address, the valid-key
+    // mask and the INT8 key scale; the ids of the next two batches and the scales of the next one are already on
+    // their way while a batch is used, so that a step costs a few shuffles and the copy request of one elected lane.
+    const int s = (warp - kLoadWarp0) & 1;
+    const bool is_v = warp >= kLoadWarp0 + 2;
+    StreamInfo S = s ? st1 : st0;
+    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
+    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
+    S.L = __shfl_sync(0xffffffffu, S.L, 0);
+    if (S.L > 0) {
+      if (!is_v && tc::elect_one()) {
+        const int nn[3] = {S.n4, S.n48 - S.n4, S.L - S.n48};
+        uint32_t bytes = 0;
+        for (int t = 0; t < 3; ++t) if (nn[t] > 0) bytes += p.qrec_bytes[t];
+        tc::mbar_arrive_expect_tx(bar(s, B_Q), bytes);
+        for (int t = 0; t < 3; ++t)
+          if (nn[t] > 0)
+            tc::bulk_g2s(smem + sm.q[s][t], p.qrec[t] + ((size_t)bh * rec_blocks(p, t) + S.a) * p.qrec_bytes[t], p.qrec_bytes[t],
+                         bar(s, B_Q));
+      }
+      __syncwarp();
+      const size_t head_blocks = (size_t)bh * R;
+      auto list_id = [&](int idx) -> int {
+        int b = idx < S.L ? (int)S.ids[idx] : 0;
+        if (b >= Rt) { atomicExch(p.status, kDevBadList); b = 0; }
+        return b;
+      };
+      auto key_scale = [&](int idx, int b) -> float {
+        return (!is_v && idx < S.L && S.tier(idx) == 1) ? p.dk8[head_blocks + b] : 0.f;
+      };
+      auto record = [&](int idx, int b) -> unsigned long long {
+        const int t = S.tier(idx);
+        return reinterpret_cast<unsigned long long>(p.kvrec[t] + ((size_t)bh * rec_blocks(p, t) + b) * p.kvrec_bytes[t] +
+                                                    (is_v ? sm.kbytes[t] : 0u));
+      };
+      int nxt_b = list_id(32 + lane), nn_b = list_id(64 + lane);
+      float cur_dk, nxt_dk = key_scale(32 + lane, nxt_b);
+      unsigned long long cur_rec, cur_mask;
+      {
+        const int b = list_id(lane);
+        cur_dk = key_scale(lane, b);
+        cur_rec = record(lane, b);
+        cur_mask = block_valid_mask(p, b);
+      }
+      const uint32_t nb0 = is_v ? sm.vbytes[0] : sm.kbytes[0], nb1 = is_v ? sm.vbytes[1] : sm.kbytes[1],
+                     nb2 = is_v ? sm.vbytes[2] : sm.kbytes[2];
+      uint8_t *dst = smem + (is_v ? sm.vst[s][0] : sm.kst[s][0]);
+      const uint32_t stage = is_v ? sm.vstage : sm.kstage;
+      const int depth = is_v ? sm.nv : sm.nk;
+      const int b_full = is_v ? B_FULLV : B_FULLK, b_free = is_v ? B_VFREE : B_KFREE;
+      int kk = 0;         // ring slot
+      uint32_t kpar = 1;  // parity of the consumption that frees the slot (first pass: nothing to wait for)
+      bool kwrapped = false;
+      for (int i = 0; i < S.L; ++i) {
+        const int src = i & 31;
+        const uint32_t rlo = __shfl_sync(0xffffffffu, (uint32_t)cur_rec, src);
+        const uint32_t rhi = __shfl_sync(0xffffffffu, (uint32_t)(cur_rec >> 32), src);
+        const uint32_t mlo = __shfl_sync(0xffffffffu, (uint32_t)cur_mask, src);
+        const uint32_t mhi = __shfl_sync(0xffffffffu, (uint32_t)(cur_mask >> 32), src);
+        const float dk = __shfl_sync(0xffffffffu, cur_dk, src);
+        const uint8_t *rec = reinterpret_cast<const uint8_t *>(((unsigned long long)rhi << 32) | rlo);
+        const uint32_t nb = i < S.n4 ? nb0 : (i < S.n48 ? nb1 : nb2);
+        if (kwrapped && !wait_or_abort(bar(s, b_free + kk), kpar, abortp)) break;
+        if (tc::elect_one()) {
+          // the step's mask and key scale enter the info ring before the data the softmax waits for is requested
+          if (!is_v)
+            *reinterpret_cast<uint4 *>(s_info + (s * kInfoRing + (i & (kInfoRing - 1))) * 16) =
+                make_uint4(mlo, mhi, __float_as_uint(dk), 0u);
+          tc::mbar_arrive_expect_tx(bar(s, b_full + kk), nb);
+          tc::bulk_g2s(dst + kk * stage, rec, nb, bar(s, b_full + kk));
+        }
+        __syncwarp();
+        if (++kk == depth) { kk = 0; kpar ^= 1u; kwrapped = true; }
+        if (src == 31) {  // next batch: its ids and scales were requested one batch ago
+          const int b = nxt_b;
+          cur_dk = nxt_dk;
+          cur_rec = record(i + 1 + lane, b);
+          cur_mask = block_valid_mask(p, b);
+          nxt_b = nn_b;
+          nxt_dk = key_scale(i + 33 + lane, nxt_b);
+          nn_b = list_id(i + 65 + lane);
+        }
+      }
+    }
+  }
+  // =========================================================================================== MMA warps
+  else if (warp >= kMmaWarp0 && warp < kPvWarp0) {
+    // The whole warp runs this loop with warp-uniform control flow and values; only the tcgen05 instructions
+    // themselves are issued by one elected lane.  (Under a lane-0 branch every descriptor would have to be moved from
+    // vector to uniform registers before each issue, which costs more than the MMA itself.)
+    const int s = warp - kMmaWarp0;
+    StreamInfo S = s ? st1 : st0;
+    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
+    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
+    S.L = __shfl_sync(0xffffffffu, S.L, 0);
+    if (S.L > 0 && wait_or_abort(bar(s, B_Q), 0, abortp)) {
+      // operand descriptors, built once; inside the loop only the 16-byte-unit start address (low bits) moves
+      const uint64_t qd0 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t qd1 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][1]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t qd2 = tc::smem_desc(tc::smem_u32(smem + sm.q[s][2]) - (s ? 1024u : 0u), 1024, 128);
+      const uint64_t kd0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]), 1024, 128);
+      const uint64_t ksf0 = tc::smem_desc(tc::smem_u32(smem + sm.kst[s][0]) + kSlots * D / 2, 128, 128);
+      const uint32_t kstep = sm.kstage >> 4;
+      const uint32_t t_sfq = tmem + col_sfq(s), t_sfk = tmem + col_sfk(s);
+      if (S.n4 > 0) {  // Q scale factors go to TMEM once; the record carries them for rows 0..63 and again for rows
+                       // 64..127, so the same atom serves either stream
+        if (tc::elect_one()) {
+#pragma unroll
+          for (int k = 0; k < D / 64; ++k)
+            tc::tmem_cp_sf(t_sfq + 4 * k, tc::smem_desc(tc::smem_u32(smem + sm.q[s][0]) + kSlots * D / 2 + k * kSfAtomBytes,
+                                                         128, 128));
+        }
+      }
+      int kk = 0;
+      uint32_t kpar = 0;
+      // the score tiles are double buffered, so Q K^T runs up to two steps ahead of the softmax
+      for (int j = 0; j < S.L; ++j) {
+        const int g = j & 1;
+        if (!wait_or_abort(bar(s, B_FULLK + kk), kpar, abortp)) break;
+        if (!wait_or_abort(bar(s, B_SFREE + g), ((j >> 1) & 1) ^ 1, abortp)) break;
+        tc::fence_after_sync();
+        const uint64_t kd = kd0 + (uint64_t)(kk * kstep);
+        const uint32_t d_s = tmem + col_s(s, g);
+        if (tc::elect_one()) {
+          if (j >= S.n48) {
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) tc::mma_f16(d_s, qd2 + ks * 128, kd + ks * 128, tc::idesc_bf16(64), ks > 0);
+          } else if (j >= S.n4) {
+#pragma unroll
+            for (int ks = 0; ks < D / 32; ++ks) tc::mma_i8(d_s, qd1 + ks * 128, kd + ks * 128, tc::idesc_i8(64), ks > 0);
+          } else {
+            const uint64_t ksf = ksf0 + (uint64_t)(kk * kstep);
+#pragma unroll
+            for (int k = 0; k < D / 64; ++k) tc::tmem_cp_sf(t_sfk + 4 * k, ksf + k * (kSfAtomBytes >> 4));
+#pragma unroll
+            for (int ks = 0; ks < D / 64; ++ks)
+              tc::mma_nvfp4(d_s, qd0 + ks * 128, kd + ks * 128, tc::idesc_nvfp4(64), ks > 0, t_sfq + 4 * ks, t_sfk + 4 * ks);
+          }
+          tc::mma_commit(bar(s, B_SREADY + (j & kMask)));
+          tc::mma_commit(bar(s, B_KFREE + kk));
+        }
+        __syncwarp();
+        if (++kk == sm.nk) { kk = 0; kpar ^= 1u; }
+      }
+    }
+  }
+  // =========================================================================================== PV warps
+  else if (warp >= kPvWarp0) {
+    const int s = warp - kPvWarp0;
+    StreamInfo S = s ? st1 : st0;
+    S.n4 = __shfl_sync(0xffffffffu, S.n4, 0);
+    S.n48 = __shfl_sync(0xffffffffu, S.n48, 0);
+    S.L = __shfl_sync(0xffffffffu, S.L, 0);
+    if (S.L > 0) {
+      const uint64_t vd0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]), D * 16, 128);
+      const uint64_t vsf0 = tc::smem_desc(tc::smem_u32(smem + sm.vst[s][0]) + D * kSlots / 2, 128, 128);
+      const uint64_t pd0 = tc::smem_desc(tc::smem_u32(smem + sm.p[s][0]), 1024, 128);
+      const uint64_t sfpd0 = tc::smem_desc(tc::smem_u32(smem + sm.sfp[s][0]), 128, 128);
+      const uint32_t pstep = sm.pbytes >> 4;
+      const uint32_t vstep = sm.vstage >> 4;
+      const uint32_t t_sfv = tmem + col_sfv(s), t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
+      int vv = 0;
+      uint32_t vpar = 0, ncorr = 0;
+      for (int j = 0; j < S.L; ++j) {
+        // ---- O^T += V(j)^T P(j)^T, once P(j) is written and the accumulator is rescaled for step j
+        const int g = j & kMask;
+        if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
+        if (!wait_or_abort(bar(s, B_PREADY + g), (j >> kShift) & 1, abortp)) break;
+        tc::fence_after_sync();
+        // The accumulator has to be rescaled before this product only if some query's maximum moved in step j or the
+        // segment changes: the step's softmax warps left the ballots in shared memory.  Only then are the stream's
+        // correction warps asked to act (they sleep on their request barrier otherwise).
+        if (j > 0) {
+          const uint2 moved = ld_shared_volatile_v2(tc::smem_u32(s_chg + (s * kSets + g) * 2));
+          if ((moved.x | moved.y) != 0u || j == S.n4 || j == S.n48) {
+            if (tc::elect_one()) {
+              s_req[s] = j;
+              tc::mbar_arrive(bar(s, B_CORRGO));
+            }
+            __syncwarp();
+            if (!wait_or_abort(bar(s, B_CORRDONE), ncorr & 1u, abortp)) break;
+            ++ncorr;
+            tc::fence_after_sync();
+          }
+        }
+        const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
+        const uint64_t pdg = pd0 + (uint64_t)(g * pstep), sfpdg = sfpd0 + (uint64_t)(g * 32);
+        const uint32_t acc = j > 0;
+        if (tc::elect_one()) {
+          if (j >= S.n48) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tc::mma_f16(t_o, vd + ks * (2 * D), pdg + ks * 128, tc::idesc_bf16(64), acc | (ks > 0));
+          } else if (j >= S.n4) {
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks)
+              tc::mma_f8f6f4(t_o, vd + ks * (2 * D), pdg + ks * 128, tc::idesc_e4m3(64), acc | (ks > 0));
+          } else {
+            tc::tmem_cp_sf(t_sfv, vsf0 + (uint64_t)(vv * vstep));
+            tc::tmem_cp_sf(t_sfp, sfpdg);
+            tc::mma_nvfp4(t_o, vd, pdg, tc::idesc_nvfp4(64), acc, t_sfv, t_sfp);
+          }
+          tc::mma_commit(bar(s, B_PVDONE + g));
+          tc::mma_commit(bar(s, B_VFREE + vv));
+        }
+        __syncwarp();
+        if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
+      }
+      if (tc::elect_one()) {  // no more requests
+        s_req[s] = -1;
+        tc::mbar_arrive(bar(s, B_CORRGO));
+      }
+      __syncwarp();
     }
   }
   // =========================================================================================== correction warps
   else {
-    const int cw = warp - kSoftmaxWarps;       // lane quarter
-    const int ch = cw * 32 + lane;             // channel (TMEM lane)
+    const int s = (warp - kSoftmaxWarps) >> 2;  // four correction warps per stream
+    const int cw = (warp - kSoftmaxWarps) & 3;  // lane quarter
+    const int ch = cw * 32 + lane;              // channel (TMEM lane)
     const uint32_t lane_addr = (uint32_t)(cw * 32) << 16;
     const float gv = p.gscale[bh * 4 + 2];
     const float dv8 = (p.tier_active[1] && ch < D) ? p.dv8[(size_t)bh * D + ch] : 0.f;
     auto unit_of = [&](int t) -> float {  // common units per accumulator unit, for this thread's channel
       return t == 0 ? __fdiv_rn(gv, 2688.0f) : (t == 1 ? kEtaP8 * dv8 : 1.0f);
     };
-    const int Lmax = max(st0.L, st1.L);
-    bool dead = false;
-    for (int i = 0; i < Lmax && !dead; ++i) {
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        const StreamInfo &S = s ? st1 : st0;
-        if (i >= S.L || dead) continue;
-        const int g = i & 1;
-        if (!wait_or_abort(bar(s, B_XREADY + g), (i >> 1) & 1, abortp)) { dead = true; continue; }
-        if (i > 0) {
-          const int tier = S.tier(i);
-          const bool tier_switch = (i == S.n4) || (i == S.n48);
-          const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * 2 + g) * 2);
-          if ((moved.x | moved.y) != 0u || tier_switch) {
-            if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abortp)) { dead = true; continue; }
-            tc::fence_after_sync();
-            float lane_factor = 1.0f;
-            if (tier_switch && ch < D) {
-              const float un = unit_of(tier), up = unit_of(S.tier(i - 1));
-              lane_factor = un > 0.f ? __fdiv_rn(up, un) : 0.f;
-            }
-            const float *fac = s_factor + (s * 2 + g) * 64;
-#pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
-              const uint32_t m8 = ((c < 4 ? moved.x : moved.y) >> ((c & 3) * 8)) & 0xffu;
-              if (m8 == 0u && !tier_switch) continue;
-              uint32_t o[8];
-              tc::tmem_ld8(tmem + lane_addr + col_o(s) + c * 8, o);
-              tc::wait_ld();
-#pragma unroll
-              for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * (fac[c * 8 + j] * lane_factor));
-              tc::tmem_st8(tmem + lane_addr + col_o(s) + c * 8, o);
-            }
-            tc::wait_st();
-            tc::fence_before_sync();
-          }
-        }
-        warp_arrive(bar(s, B_PREADY + g));
+    const StreamInfo &S = s ? st1 : st0;
+    // requests from the stream's product-issuing warp: "rescale the accumulator for step i"; -1 ends the loop
+    for (uint32_t nreq = 0; S.L > 0; ++nreq) {
+      if (!wait_or_abort(bar(s, B_CORRGO), nreq & 1u, abortp)) break;
+      const int i = *reinterpret_cast<volatile int *>(&s_req[s]);
+      if (i < 0) break;
+      const int g = i & kMask;
+      const int tier = S.tier(i);
+      const bool tier_switch = (i == S.n4) || (i == S.n48);
+      const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * kSets + g) * 2);
+      if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & kMask)), ((i - 1) >> kShift) & 1, abortp)) break;
+      tc::fence_after_sync();
+      float lane_factor = 1.0f;
+      if (tier_switch && ch < D) {
+        const float un = unit_of(tier), up = unit_of(S.tier(i - 1));
+        lane_factor = un > 0.f ? __fdiv_rn(up, un) : 0.f;
       }
+      const float *fac = s_factor + (s * kSets + g) * 64;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t m8 = ((c < 4 ? moved.x : moved.y) >> ((c & 3) * 8)) & 0xffu;
+        if (m8 == 0u && !tier_switch) continue;
+        uint32_t o[8];
+        tc::tmem_ld8(tmem + lane_addr + col_o(s) + c * 8, o);
+        tc::wait_ld();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * (fac[c * 8 + j] * lane_factor));
+        tc::tmem_st8(tmem + lane_addr + col_o(s) + c * 8, o);
+      }
+      tc::wait_st();
+      tc::fence_before_sync();
+      warp_arrive(bar(s, B_CORRDONE));
     }
     // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
-#pragma unroll
-    for (int s = 0; s < 2; ++s) {
-      const StreamInfo &S = s ? st1 : st0;
-      if (S.a < 0) continue;
+    if (S.a >= 0) {
       const unsigned long long qmask = block_valid_mask(p, S.a);
       uint16_t *stage = reinterpret_cast<uint16_t *>(smem + sm.kst[s][0]);  // [64][D] bf16 over the K ring
       bool ok = S.L > 0 && !*abortp;
       if (ok) ok = wait_or_abort(bar(s, B_ELL), 0, abortp);
-      if (ok) ok = wait_or_abort(bar(s, B_PVDONE + ((S.L - 1) & 1)), ((S.L - 1) >> 1) & 1, abortp);
+      if (ok) ok = wait_or_abort(bar(s, B_PVDONE + ((S.L - 1) & kMask)), ((S.L - 1) >> kShift) & 1, abortp);
       if (ok) {
         tc::fence_after_sync();
         const float unit = ch < D ? unit_of(S.tier(S.L - 1)) : 0.f;
@@ -826,20 +898,26 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
             for (int j = 0; j < 8; ++j) {
               const int qr = c * 8 + j;
               // the two warps of a row kept partial denominators relative to their own last maximum
-              const float h0 = s_xmax[((s * 2 + 0) * 2 + 1) * 64 + qr], h1 = s_xmax[((s * 2 + 1) * 2 + 1) * 64 + qr];
-              const float hf = fmaxf(h0, h1);
-              const float l = s_ell[(s * 2 + 0) * 64 + qr] * ex2(h0 - hf) + s_ell[(s * 2 + 1) * 64 + qr] * ex2(h1 - hf);
+              float hf = -INFINITY, l = 0.f;
+#pragma unroll
+              for (int k = 0; k < kSets; ++k) hf = fmaxf(hf, s_href[(s * kSets + k) * 64 + qr]);
+#pragma unroll
+              for (int k = 0; k < kSets; ++k) {  // a set without a step has ell = 0 and reference -inf
+                const float lk = s_ell[(s * kSets + k) * 64 + qr];
+                if (lk > 0.f) l += lk * ex2(s_href[(s * kSets + k) * 64 + qr] - hf);
+              }
               const float val = l > 0.f ? __uint_as_float(o[j]) * unit * __fdiv_rn(1.0f, l) : 0.f;
               stage[qr * D + ch] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
             }
           }
         }
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int ltid = tid - (kSoftmaxWarps + 4 * s) * 32;  // thread index inside the stream's correction group
+      if (s == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
       if (S.L == 0) {
-        store_zero_rows(S.a, tid - kSoftmaxWarps * 32, kCorrWarps * 32);
+        store_zero_rows(S.a, ltid, 128);
       } else if (ok) {
-        for (int idx = tid - kSoftmaxWarps * 32; idx < kSlots * (D / 8); idx += kCorrWarps * 32) {
+        for (int idx = ltid; idx < kSlots * (D / 8); idx += 128) {
           const int j = idx / (D / 8), c8 = idx % (D / 8);
           if ((qmask >> j) & 1ull)
             *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, S.a, j) * D + c8 * 8) =
@@ -848,6 +926,8 @@ __global__ void __launch_bounds__(NT, 1) attention_kernel(Params p, SmemMap sm, 
       }
     }
   }
+
+  }  // warps without a score row
 
   tc::fence_before_sync();
   __syncthreads();
@@ -887,26 +967,39 @@ cudaError_t launch_bounded_wait_probe(int *status, long long limit_cycles, cudaS
 }
 
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches) {
-  const SmemMap sm = make_smem_map(p);
+  // four softmax sets when their P images leave room for rings of at least 2 K and 3 V stages, else two
+  SmemMap sm = make_smem_map(p, 4);
+  int sets = 4;
+  if (!sm.fits || sm.nv < 3) {
+    sm = make_smem_map(p, 2);
+    sets = 2;
+  }
+  if (!sm.fits) return cudaErrorInvalidConfiguration;
   cudaError_t e;
   const int grid = p.BH * ((p.Rt + 1) / 2);
-  auto launch = [&](auto kernel) -> cudaError_t {
+  auto launch = [&](auto kernel, int nt) -> cudaError_t {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total);
     if (err != cudaSuccess) return err;
-    kernel<<<grid, NT, sm.total, st>>>(p, sm, out);
+    kernel<<<grid, nt, sm.total, st>>>(p, sm, out);
     return cudaSuccess;
   };
   const bool ordered = p.rank_scope != 0, fp4 = p.tier_active[0] != 0;
-  if (p.d == 128) {
-    e = ordered ? (fp4 ? launch(attention_kernel<128, true, true>) : launch(attention_kernel<128, true, false>))
-                : (fp4 ? launch(attention_kernel<128, false, true>) : launch(attention_kernel<128, false, false>));
-  } else {
-    e = ordered ? (fp4 ? launch(attention_kernel<64, true, true>) : launch(attention_kernel<64, true, false>))
-                : (fp4 ? launch(attention_kernel<64, false, true>) : launch(attention_kernel<64, false, false>));
-  }
+  auto pick = [&](auto dtag, auto stag) -> cudaError_t {
+    constexpr int D = decltype(dtag)::value, S = decltype(stag)::value;
+    constexpr int nt = Roles<S>::NT;
+    return ordered ? (fp4 ? launch(attention_kernel<D, true, true, S>, nt) : launch(attention_kernel<D, true, false, S>, nt))
+                   : (fp4 ? launch(attention_kernel<D, false, true, S>, nt) : launch(attention_kernel<D, false, false, S>, nt));
+  };
+  using I64 = std::integral_constant<int, 64>;
+  using I128 = std::integral_constant<int, 128>;
+  using S2 = std::integral_constant<int, 2>;
+  using S4 = std::integral_constant<int, 4>;
+  if (p.d == 128) e = sets == 4 ? pick(I128{}, S4{}) : pick(I128{}, S2{});
+  else e = sets == 4 ? pick(I64{}, S4{}) : pick(I64{}, S2{});
   if (e != cudaSuccess) return e;
   *launches += 1;
   return cudaGetLastError();
 }
 
 }  // namespace da2
+
