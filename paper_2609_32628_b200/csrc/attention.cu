@@ -14,13 +14,14 @@
 //                     of step i-1 from the thread of the previous set through a shared-memory word tagged with the
 //                     step, keeps a partial denominator, and writes P~ (and its NVFP4 scale factors) into its set's
 //                     operand image.  These warps hold most of the register file (setmaxnreg).
-//     next 8 warps    correction + epilogue, four per stream: rescale the accumulator columns of queries whose
-//                     maximum moved and apply the per-channel unit change at a segment boundary ON REQUEST of the
-//                     PV-issue warp (most steps move no maximum and request nothing), and finally combine the sets'
-//                     partial denominators, normalise, transpose and store
+//     next 8 warps    correction + epilogue, four per stream.  Every step passes through them between the softmax
+//                     and the product: they read the step's "maximum moved" ballots and, only if one is set or the
+//                     segment changes, wait for the previous product and rescale those accumulator columns (and apply
+//                     the per-channel unit change); then they release the product.  Most steps move no maximum, and
+//                     the check is off the issuing warp's instruction stream.  Finally they combine the sets' partial
+//                     denominators, normalise, transpose and store
 //     next 2 warps    S = Q K^T issue, one warp per stream (tcgen05.mma, accumulators in TMEM), two steps ahead
-//     next 2 warps    O^T += V^T P~^T issue, one warp per stream; reads the step's "maximum moved" ballots and asks
-//                     for a correction only when one is set or the tier changes.  The issuing warps' instruction
+//     next 2 warps    O^T += V^T P~^T issue, one warp per stream.  The issuing warps' instruction
 //                     counts are on the critical path of every step: their loops are warp-uniform (one elected lane
 //                     issues), operand descriptors are built once and only offset inside the loop
 //     last 4 warps    loaders: per stream one warp for K (and the Q records) and one for V^T, 1-D bulk copies into
@@ -82,8 +83,7 @@ constexpr float kOffsetP8 = 8.807f;      // base-2 exponent offset (about log2 4
 // barrier indices inside one stream's group
 // (a parity wait can only tell the latest completion from the one before, so every barrier is laid out such that no
 // waiter can fall two completions behind: buffers indexed by step parity get one barrier per buffer)
-enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 10, B_VFREE = 14, B_SREADY = 20, B_SFREE = 24, B_PREADY = 26, B_CORRGO = 30,
-       B_CORRDONE = 31, B_PVDONE = 34, B_ELL = 38, B_Q = 39, B_COUNT = 40 };
+enum { B_FULLK = 0, B_FULLV = 4, B_KFREE = 10, B_VFREE = 14, B_SREADY = 20, B_SFREE = 24, B_PREADY = 26, B_CORROK = 30, B_PVDONE = 34, B_ELL = 38, B_Q = 39, B_COUNT = 40 };
 constexpr int kMaxK = 4, kMaxV = 6, kInfoRing = 8;
 
 struct SmemMap {
@@ -300,7 +300,6 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ int s_req[2];  // step a stream's correction warps are asked to rescale for
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
@@ -351,6 +350,7 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         tc::mbar_init(bar(s, B_SREADY + g), 1);
         tc::mbar_init(bar(s, B_PREADY + g), 2);  // the two softmax warps of the step (P written)
         tc::mbar_init(bar(s, B_PVDONE + g), 1);
+        tc::mbar_init(bar(s, B_CORROK + g), 4);  // the stream's four correction warps (accumulator rescaled)
       }
       for (int g = 0; g < kMaxK; ++g) {
         tc::mbar_init(bar(s, B_FULLK + g), 1);
@@ -361,8 +361,6 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         tc::mbar_init(bar(s, B_VFREE + g), 1);
       }
       tc::mbar_init(bar(s, B_ELL), 2 * kSets);
-      tc::mbar_init(bar(s, B_CORRGO), 1);
-      tc::mbar_init(bar(s, B_CORRDONE), 4);
       tc::mbar_init(bar(s, B_Q), 1);
     }
     tc::fence_barrier_init();
@@ -467,7 +465,7 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         }
         const bool got = hv.y == (uint32_t)(i - 1);
         if (!__all_sync(0xffffffffu, got)) {
-          atomicCAS(const_cast<int *>(abortp), 0, 1 + (int)(tc::smem_u32(bar(s, B_CORRGO)) & 0xffff));
+          atomicCAS(const_cast<int *>(abortp), 0, 1 + (int)(tc::smem_u32(bar(s, B_CORROK)) & 0xffff));
           break;
         }
         h_prev = __uint_as_float(hv.x);
@@ -781,29 +779,14 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
       const uint32_t vstep = sm.vstage >> 4;
       const uint32_t t_sfv = tmem + col_sfv(s), t_sfp = tmem + col_sfp(s), t_o = tmem + col_o(s);
       int vv = 0;
-      uint32_t vpar = 0, ncorr = 0;
+      uint32_t vpar = 0;
       for (int j = 0; j < S.L; ++j) {
         // ---- O^T += V(j)^T P(j)^T, once P(j) is written and the accumulator is rescaled for step j
         const int g = j & kMask;
         if (!wait_or_abort(bar(s, B_FULLV + vv), vpar, abortp)) break;
-        if (!wait_or_abort(bar(s, B_PREADY + g), (j >> kShift) & 1, abortp)) break;
+        // P(j) is written and the stream's correction warps have rescaled the accumulator where step j asked for it
+        if (!wait_or_abort(bar(s, B_CORROK + g), (j >> kShift) & 1, abortp)) break;
         tc::fence_after_sync();
-        // The accumulator has to be rescaled before this product only if some query's maximum moved in step j or the
-        // segment changes: the step's softmax warps left the ballots in shared memory.  Only then are the stream's
-        // correction warps asked to act (they sleep on their request barrier otherwise).
-        if (j > 0) {
-          const uint2 moved = ld_shared_volatile_v2(tc::smem_u32(s_chg + (s * kSets + g) * 2));
-          if ((moved.x | moved.y) != 0u || j == S.n4 || j == S.n48) {
-            if (tc::elect_one()) {
-              s_req[s] = j;
-              tc::mbar_arrive(bar(s, B_CORRGO));
-            }
-            __syncwarp();
-            if (!wait_or_abort(bar(s, B_CORRDONE), ncorr & 1u, abortp)) break;
-            ++ncorr;
-            tc::fence_after_sync();
-          }
-        }
         const uint64_t vd = vd0 + (uint64_t)(vv * vstep);
         const uint64_t pdg = pd0 + (uint64_t)(g * pstep), sfpdg = sfpd0 + (uint64_t)(g * 32);
         const uint32_t acc = j > 0;
@@ -827,11 +810,6 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         __syncwarp();
         if (++vv == sm.nv) { vv = 0; vpar ^= 1u; }
       }
-      if (tc::elect_one()) {  // no more requests
-        s_req[s] = -1;
-        tc::mbar_arrive(bar(s, B_CORRGO));
-      }
-      __syncwarp();
     }
   }
   // =========================================================================================== correction warps
@@ -846,15 +824,19 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
       return t == 0 ? __fdiv_rn(gv, 2688.0f) : (t == 1 ? kEtaP8 * dv8 : 1.0f);
     };
     const StreamInfo &S = s ? st1 : st0;
-    // requests from the stream's product-issuing warp: "rescale the accumulator for step i"; -1 ends the loop
-    for (uint32_t nreq = 0; S.L > 0; ++nreq) {
-      if (!wait_or_abort(bar(s, B_CORRGO), nreq & 1u, abortp)) break;
-      const int i = *reinterpret_cast<volatile int *>(&s_req[s]);
-      if (i < 0) break;
+    // Every step passes through these warps between the softmax and the product: once P(i) is written they read the
+    // step's "maximum moved" ballots and, only if one is set or the segment changes, wait for product i-1 and rescale
+    // their lane quarter of the accumulator; then they let product i go.  Most steps move no maximum.
+    for (int i = 0; i < S.L; ++i) {
       const int g = i & kMask;
-      const int tier = S.tier(i);
+      if (!wait_or_abort(bar(s, B_PREADY + g), (i >> kShift) & 1, abortp)) break;
       const bool tier_switch = (i == S.n4) || (i == S.n48);
-      const uint2 moved = *reinterpret_cast<const uint2 *>(s_chg + (s * kSets + g) * 2);
+      const uint2 moved = ld_shared_volatile_v2(tc::smem_u32(s_chg + (s * kSets + g) * 2));
+      if (i == 0 || ((moved.x | moved.y) == 0u && !tier_switch)) {
+        if (lane == 0) tc::mbar_arrive(bar(s, B_CORROK + g));
+        continue;
+      }
+      const int tier = S.tier(i);
       if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & kMask)), ((i - 1) >> kShift) & 1, abortp)) break;
       tc::fence_after_sync();
       float lane_factor = 1.0f;
@@ -876,7 +858,7 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
       }
       tc::wait_st();
       tc::fence_before_sync();
-      warp_arrive(bar(s, B_CORRDONE));
+      warp_arrive(bar(s, B_CORROK + g));
     }
     // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
     if (S.a >= 0) {
