@@ -267,6 +267,20 @@ __device__ __forceinline__ uint2 ld_shared_volatile_v2(uint32_t saddr) {
   return r;
 }
 
+// Valid-slot mask and token index of a block, from the frame's region table (prefix blocks are runs of 64 tokens)
+__device__ __forceinline__ unsigned long long table_mask(const Params &p, int a) {
+  if (a >= p.R) {
+    const int rem = p.P - (a - p.R) * kSlots;
+    return rem >= kSlots ? ~0ull : ((1ull << rem) - 1ull);
+  }
+  return p.region_mask[a % p.R_f];
+}
+__device__ __forceinline__ long long table_token(const Params &p, int a, int j) {
+  if (a >= p.R) return (long long)(a - p.R) * kSlots + j;
+  const int t = a / p.R_f, r = a - t * p.R_f;
+  return p.P + (long long)t * (p.Hg * p.Wg) + p.region_cell[r * kSlots + j];
+}
+
 struct StreamInfo {
   int a;         // query block, or -1
   int n4, n48;   // end of the NVFP4 segment, end of the INT8 segment (list positions)
@@ -314,20 +328,6 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
     a1 = ord[1];
   }
   const StreamInfo st0 = load_stream(p, bh, a0), st1 = load_stream(p, bh, a1);
-
-  auto store_zero_rows = [&](int a, int first, int nthreads) {  // rows without a retained key return zero (App. C.1)
-    const unsigned long long qmask = block_valid_mask(p, a);
-    for (int idx = first; idx < kSlots * (D / 8); idx += nthreads) {
-      const int j = idx / (D / 8), c8 = idx % (D / 8);
-      if ((qmask >> j) & 1ull)
-        *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, a, j) * D + c8 * 8) = make_uint4(0, 0, 0, 0);
-    }
-  };
-  if (st0.L == 0 && st1.L == 0) {
-    if (st0.a >= 0) store_zero_rows(st0.a, tid, NT);
-    if (st1.a >= 0) store_zero_rows(st1.a, tid, NT);
-    return;
-  }
 
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + sm.bars);
   auto bar = [&](int s, int which) -> uint64_t * { return bars + s * B_COUNT + which; };
@@ -652,15 +652,10 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         return reinterpret_cast<unsigned long long>(p.kvrec[t] + ((size_t)bh * rec_blocks(p, t) + b) * p.kvrec_bytes[t] +
                                                     (is_v ? sm.kbytes[t] : 0u));
       };
-      int nxt_b = list_id(32 + lane), nn_b = list_id(64 + lane);
-      float cur_dk, nxt_dk = key_scale(32 + lane, nxt_b);
-      unsigned long long cur_rec, cur_mask;
-      {
-        const int b = list_id(lane);
-        cur_dk = key_scale(lane, b);
-        cur_rec = record(lane, b);
-        cur_mask = block_valid_mask(p, b);
-      }
+      // batch -1 is empty: the loop's refill at "src == 31" then also serves the first batch
+      int nxt_b = list_id(lane), nn_b = list_id(32 + lane);
+      float cur_dk = 0.f, nxt_dk = key_scale(lane, nxt_b);
+      unsigned long long cur_rec = 0, cur_mask = 0;
       const uint32_t nb0 = is_v ? sm.vbytes[0] : sm.kbytes[0], nb1 = is_v ? sm.vbytes[1] : sm.kbytes[1],
                      nb2 = is_v ? sm.vbytes[2] : sm.kbytes[2];
       uint8_t *dst = smem + (is_v ? sm.vst[s][0] : sm.kst[s][0]);
@@ -670,8 +665,9 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
       int kk = 0;         // ring slot
       uint32_t kpar = 1;  // parity of the consumption that frees the slot (first pass: nothing to wait for)
       bool kwrapped = false;
-      for (int i = 0; i < S.L; ++i) {
+      for (int i = -1; i < S.L; ++i) {
         const int src = i & 31;
+        if (i >= 0) {
         const uint32_t rlo = __shfl_sync(0xffffffffu, (uint32_t)cur_rec, src);
         const uint32_t rhi = __shfl_sync(0xffffffffu, (uint32_t)(cur_rec >> 32), src);
         const uint32_t mlo = __shfl_sync(0xffffffffu, (uint32_t)cur_mask, src);
@@ -690,11 +686,12 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         }
         __syncwarp();
         if (++kk == depth) { kk = 0; kpar ^= 1u; kwrapped = true; }
+        }
         if (src == 31) {  // next batch: its ids and scales were requested one batch ago
           const int b = nxt_b;
           cur_dk = nxt_dk;
           cur_rec = record(i + 1 + lane, b);
-          cur_mask = block_valid_mask(p, b);
+          cur_mask = table_mask(p, b);
           nxt_b = nn_b;
           nxt_dk = key_scale(i + 33 + lane, nxt_b);
           nn_b = list_id(i + 65 + lane);
@@ -862,11 +859,26 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
     }
     // ---------------------------------------------------------- epilogue: O = U / l, back to raster order
     if (S.a >= 0) {
-      const unsigned long long qmask = block_valid_mask(p, S.a);
+      const unsigned long long qmask = table_mask(p, S.a);
       uint16_t *stage = reinterpret_cast<uint16_t *>(smem + sm.kst[s][0]);  // [64][D] bf16 over the K ring
       bool ok = S.L > 0 && !*abortp;
       if (ok) ok = wait_or_abort(bar(s, B_ELL), 0, abortp);
       if (ok) ok = wait_or_abort(bar(s, B_PVDONE + ((S.L - 1) & kMask)), ((S.L - 1) >> kShift) & 1, abortp);
+      const int ltid = tid - (kSoftmaxWarps + 4 * s) * 32;  // thread index inside the stream's correction group
+      float *s_inv = s_factor + (s * kSets) * 64;            // 1 / l per query (the factors are no longer needed)
+      if (ok && ltid < 64) {
+        // the sets of a row kept partial denominators relative to their own last maximum
+        float hf = -INFINITY, l = 0.f;
+#pragma unroll 1
+        for (int k = 0; k < kSets; ++k) hf = fmaxf(hf, s_href[(s * kSets + k) * 64 + ltid]);
+#pragma unroll 1
+        for (int k = 0; k < kSets; ++k) {  // a set without a step has ell = 0 and reference -inf
+          const float lk = s_ell[(s * kSets + k) * 64 + ltid];
+          if (lk > 0.f) l += lk * ex2(s_href[(s * kSets + k) * 64 + ltid] - hf);
+        }
+        s_inv[ltid] = l > 0.f ? __fdiv_rn(1.0f, l) : 0.f;
+      }
+      if (s == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
       if (ok) {
         tc::fence_after_sync();
         const float unit = ch < D ? unit_of(S.tier(S.L - 1)) : 0.f;
@@ -879,30 +891,22 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const int qr = c * 8 + j;
-              // the two warps of a row kept partial denominators relative to their own last maximum
-              float hf = -INFINITY, l = 0.f;
-#pragma unroll
-              for (int k = 0; k < kSets; ++k) hf = fmaxf(hf, s_href[(s * kSets + k) * 64 + qr]);
-#pragma unroll
-              for (int k = 0; k < kSets; ++k) {  // a set without a step has ell = 0 and reference -inf
-                const float lk = s_ell[(s * kSets + k) * 64 + qr];
-                if (lk > 0.f) l += lk * ex2(s_href[(s * kSets + k) * 64 + qr] - hf);
-              }
-              const float val = l > 0.f ? __uint_as_float(o[j]) * unit * __fdiv_rn(1.0f, l) : 0.f;
+              const float inv = s_inv[qr];
+              const float val = inv > 0.f ? __uint_as_float(o[j]) * unit * inv : 0.f;
               stage[qr * D + ch] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
             }
           }
         }
+      } else if (S.L == 0) {  // rows without a retained key return zero (App. C.1)
+        for (int idx = ltid; idx < kSlots * (D / 8); idx += 128) reinterpret_cast<uint4 *>(stage)[idx] = make_uint4(0, 0, 0, 0);
       }
-      const int ltid = tid - (kSoftmaxWarps + 4 * s) * 32;  // thread index inside the stream's correction group
       if (s == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
-      if (S.L == 0) {
-        store_zero_rows(S.a, ltid, 128);
-      } else if (ok) {
+      if (ok || S.L == 0) {
+#pragma unroll 1
         for (int idx = ltid; idx < kSlots * (D / 8); idx += 128) {
           const int j = idx / (D / 8), c8 = idx % (D / 8);
           if ((qmask >> j) & 1ull)
-            *reinterpret_cast<uint4 *>(out_head + (size_t)slot_token(p, S.a, j) * D + c8 * 8) =
+            *reinterpret_cast<uint4 *>(out_head + (size_t)table_token(p, S.a, j) * D + c8 * 8) =
                 *reinterpret_cast<const uint4 *>(stage + j * D + c8 * 8);
         }
       }

@@ -73,6 +73,8 @@ da2::Params make_params(const da2_plan_t *plan, void *workspace) {
   p.dq8 = (float *)(w + I.off_dq8);
   p.dk8 = (float *)(w + I.off_dk8);
   p.dv8 = (float *)(w + I.off_dv8);
+  p.region_cell = (int *)(w + plan->off_region_cell);
+  p.region_mask = (unsigned long long *)(w + plan->off_region_mask);
   return p;
 }
 
@@ -244,6 +246,8 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   I.off_dk8 = c.take(BH * R * 4);
   I.off_dv8 = c.take(BH * d * 4);
   I.off_order = c.take(BH * (uint64_t)(2 * ((R + 1) / 2)) * 2);
+  plan->off_region_cell = c.take((uint64_t)I.R_f * da2::kSlots * 4);
+  plan->off_region_mask = c.take((uint64_t)I.R_f * 8);
   I.workspace_bytes = c.cur;
 
   const float *src[3] = {cfg->g_q, cfg->g_k, cfg->g_v};

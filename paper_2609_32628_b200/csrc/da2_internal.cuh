@@ -49,6 +49,10 @@ struct Params {
   uint8_t *qrec[3], *kvrec[3];
   float *dq8, *dk8, *dv8;
   uint16_t *order;          // [BH][2*ceil(R/2)] query blocks by decreasing list length
+  // region table of one frame, written with the operand records: cell (y * Wg + x) of slot j of region r, and the
+  // region's slot-valid mask; the attention kernel looks tokens up here instead of carrying the region arithmetic
+  int *region_cell;               // [R_f][64]
+  unsigned long long *region_mask;  // [R_f]
 };
 
 // number of valid rows / columns of tile (ty, tx) and the 64-bit slot-valid mask of block a
@@ -121,4 +125,5 @@ struct da2_plan {
   da2_config_t cfg;
   da2_plan_info_t info;
   float *g_host[3];       // optional caller-provided NVFP4 per-tensor scales (copied), or nullptr
+  uint64_t off_region_cell, off_region_mask;  // workspace offsets of the region table (internal)
 };

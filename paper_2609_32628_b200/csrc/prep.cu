@@ -75,6 +75,11 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
   const size_t blk = (size_t)bh * p.R + a;        // record index in the quantised tiers (video blocks only)
   const size_t blk16 = (size_t)bh * p.Rt + a;     // record index in the 16-bit tier (video and prefix blocks)
   const bool video = a < p.R;                      // prefix blocks only ever run in the 16-bit tier (App. C.1)
+  // the regions of the first frame also leave the frame's region table for the attention kernel
+  if (bh == 0 && a < p.R_f) {
+    if (tid < kSlots) p.region_cell[a * kSlots + tid] = (int)(slot_token(p, a, tid) - p.P);
+    if (tid == 0) p.region_mask[a] = mask;
+  }
 
   // stage the three tiles, padding slots as zeros; track max|Q|, max|K| of the block
   float aq = 0.f, ak = 0.f;
