@@ -20,6 +20,11 @@ constexpr int NT = 256;
 
 __device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
 
+// round half away from zero for |x| < 2^23: adding the largest float below one half (with the sign of x) and truncating
+// gives the same integer as roundf for every x in that range (the sum can only round up to the next integer when x
+// is at least one half above the integer below it)
+__device__ __forceinline__ int round_half_away(float x) { return __float2int_rz(__fadd_rn(x, copysignf(0x1.fffffep-2f, x))); }
+
 __device__ __forceinline__ uint32_t cast_e4m3(float x) {
   return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
 }
@@ -90,9 +95,11 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
                                                   const __nv_bfloat16 *__restrict__ v) {
   extern __shared__ __align__(16) uint8_t smem[];
   uint16_t *tq = reinterpret_cast<uint16_t *>(smem);   // [64][D]
-  uint16_t *tk = tq + kSlots * D;
-  uint16_t *tv = tk + kSlots * D;
-  uint8_t *sf_img = reinterpret_cast<uint8_t *>(tv + kSlots * D);  // up to 3 atoms (Q or K: D/64, V: 1)
+  // rows are padded by 16 bytes: threads that read the same channels of consecutive slots then fall on different banks
+  constexpr int LD = D + 8;
+  uint16_t *tk = tq + kSlots * LD;
+  uint16_t *tv = tk + kSlots * LD;
+  uint8_t *sf_img = reinterpret_cast<uint8_t *>(tv + kSlots * LD);  // up to 3 atoms (Q or K: D/64, V: 1)
   __shared__ float s_red[2][NT / 32];
   __shared__ float s_delta[2];
 
@@ -120,9 +127,9 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
       xk = *reinterpret_cast<const uint4 *>(k + off);
       xv = *reinterpret_cast<const uint4 *>(v + off);
     }
-    *reinterpret_cast<uint4 *>(tq + j * D + c8 * 8) = xq;
-    *reinterpret_cast<uint4 *>(tk + j * D + c8 * 8) = xk;
-    *reinterpret_cast<uint4 *>(tv + j * D + c8 * 8) = xv;
+    *reinterpret_cast<uint4 *>(tq + j * LD + c8 * 8) = xq;
+    *reinterpret_cast<uint4 *>(tk + j * LD + c8 * 8) = xk;
+    *reinterpret_cast<uint4 *>(tv + j * LD + c8 * 8) = xv;
     const uint32_t wq[4] = {xq.x, xq.y, xq.z, xq.w}, wk[4] = {xk.x, xk.y, xk.z, xk.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -158,7 +165,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 #pragma unroll 8
       for (int j = 0; j < kSlots; ++j) {
         if ((mask >> j) & 1ull) {
-          const float x = bf16_to_f32(src[j * D]);
+          const float x = bf16_to_f32(src[j * LD]);
           sum += (double)x;
           mx = fmaxf(mx, x);
         }
@@ -176,15 +183,15 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
     uint8_t *vr = kr + kSlots * D * 2;
     for (int idx = tid; idx < kSlots * D / 8; idx += NT) {  // chunk (kc, r): channels kc*8.. of slot r
       const int kc = idx / kSlots, r = idx % kSlots;
-      *reinterpret_cast<uint4 *>(qr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tq + r * D + kc * 8);
-      *reinterpret_cast<uint4 *>(kr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tk + r * D + kc * 8);
+      *reinterpret_cast<uint4 *>(qr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tq + r * LD + kc * 8);
+      *reinterpret_cast<uint4 *>(kr + (size_t)idx * 16) = *reinterpret_cast<const uint4 *>(tk + r * LD + kc * 8);
     }
     for (int idx = tid; idx < D * kSlots / 8; idx += NT) {  // chunk (kc, c): slots kc*8.. of channel c
       const int kc = idx / D, c = idx % D;
       uint32_t w[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        w[i] = (uint32_t)tv[(kc * 8 + 2 * i) * D + c] | ((uint32_t)tv[(kc * 8 + 2 * i + 1) * D + c] << 16);
+        w[i] = (uint32_t)tv[(kc * 8 + 2 * i) * LD + c] | ((uint32_t)tv[(kc * 8 + 2 * i + 1) * LD + c] << 16);
       *reinterpret_cast<uint4 *>(vr + (size_t)idx * 16) = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
@@ -199,16 +206,16 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
       const int kc = idx / kSlots, r = idx % kSlots;
       uint32_t wq[4] = {0, 0, 0, 0}, wk[4] = {0, 0, 0, 0};
       uint32_t xq[8], xk[8];  // 16 bf16 values each, two per word
-      *reinterpret_cast<uint4 *>(xq) = *reinterpret_cast<const uint4 *>(tq + r * D + kc * 16);
-      *reinterpret_cast<uint4 *>(xq + 4) = *reinterpret_cast<const uint4 *>(tq + r * D + kc * 16 + 8);
-      *reinterpret_cast<uint4 *>(xk) = *reinterpret_cast<const uint4 *>(tk + r * D + kc * 16);
-      *reinterpret_cast<uint4 *>(xk + 4) = *reinterpret_cast<const uint4 *>(tk + r * D + kc * 16 + 8);
+      *reinterpret_cast<uint4 *>(xq) = *reinterpret_cast<const uint4 *>(tq + r * LD + kc * 16);
+      *reinterpret_cast<uint4 *>(xq + 4) = *reinterpret_cast<const uint4 *>(tq + r * LD + kc * 16 + 8);
+      *reinterpret_cast<uint4 *>(xk) = *reinterpret_cast<const uint4 *>(tk + r * LD + kc * 16);
+      *reinterpret_cast<uint4 *>(xk + 4) = *reinterpret_cast<const uint4 *>(tk + r * LD + kc * 16 + 8);
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const float fq = __uint_as_float((i & 1) ? (xq[i >> 1] & 0xffff0000u) : (xq[i >> 1] << 16));
         const float fk = __uint_as_float((i & 1) ? (xk[i >> 1] & 0xffff0000u) : (xk[i >> 1] << 16));
-        const int cq = (int)roundf(dq.fast ? dq.quick(fq) : dq.exact(fq));
-        const int ck = (int)roundf(dk.fast ? dk.quick(fk) : dk.exact(fk));
+        const int cq = round_half_away(dq.fast ? dq.quick(fq) : dq.exact(fq));
+        const int ck = round_half_away(dk.fast ? dk.quick(fk) : dk.exact(fk));
         wq[i >> 2] |= (uint32_t)(cq & 0xff) << (8 * (i & 3));
         wk[i >> 2] |= (uint32_t)(ck & 0xff) << (8 * (i & 3));
       }
@@ -225,13 +232,13 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
         if (div.fast) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const uint32_t code = cast_e4m3(div.quick(bf16_to_f32(tv[(kc * 16 + i) * D + c])));
+            const uint32_t code = cast_e4m3(div.quick(bf16_to_f32(tv[(kc * 16 + i) * LD + c])));
             w[i >> 2] |= ((m16 >> i) & 1u) ? code << (8 * (i & 3)) : 0u;
           }
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const uint32_t code = cast_e4m3(div.exact(bf16_to_f32(tv[(kc * 16 + i) * D + c])));
+            const uint32_t code = cast_e4m3(div.exact(bf16_to_f32(tv[(kc * 16 + i) * LD + c])));
             w[i >> 2] |= ((m16 >> i) & 1u) ? code << (8 * (i & 3)) : 0u;
           }
         }
@@ -262,7 +269,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
           float x[16];
           uint32_t pk[2];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(src[r * D + kc * 32 + h * 16 + i]);
+          for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(src[r * LD + kc * 32 + h * 16 + i]);
           const uint32_t sc = nvfp4_group(x, g, pk);
           w[2 * h] = pk[0]; w[2 * h + 1] = pk[1];
           const int grp = kc * 2 + h;  // 16-channel group index; 4 groups per atom
@@ -288,7 +295,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
         float x[16];
         uint32_t pk[2];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(tv[(kc * 32 + h * 16 + i) * D + c]);
+        for (int i = 0; i < 16; ++i) x[i] = bf16_to_f32(tv[(kc * 32 + h * 16 + i) * LD + c]);
         const uint32_t sc = nvfp4_group(x, gv, pk);
         w[2 * h] = pk[0]; w[2 * h + 1] = pk[1];
         sf_img[(c & 31) * 16 + (c >> 5) * 4 + (kc * 2 + h)] = (uint8_t)sc;
@@ -306,7 +313,7 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches, bool pool) {
   dim3 grid(p.Rt, p.BH);
-  const size_t smem = 3 * (size_t)kSlots * p.d * 2 + 3 * kSfAtomBytes;
+  const size_t smem = 3 * (size_t)kSlots * (p.d + 8) * 2 + 3 * kSfAtomBytes;
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
