@@ -37,16 +37,23 @@ __global__ void __launch_bounds__(256) pool_kernel(Params p, const __nv_bfloat16
 #pragma unroll
   for (int i = 0; i < 8; ++i) { sq[i] = 0.0; sk[i] = 0.0; mq[i] = -INFINITY; mk[i] = -INFINITY; av[i] = 0.f; }
 
+  // all loads of the thread are issued before the first is used (a padding slot reads slot 0's row and is ignored)
+  uint4 xq[PASSES], xk[PASSES], xv[PASSES];
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int j = ps * TP + tsub;
+    const int js = ((mask >> j) & 1ull) ? j : 0;
+    const size_t off = head_off + (size_t)slot_token(p, a, js) * D + cidx * 8;
+    xq[ps] = *reinterpret_cast<const uint4 *>(q + off);
+    xk[ps] = *reinterpret_cast<const uint4 *>(k + off);
+    xv[ps] = *reinterpret_cast<const uint4 *>(v + off);
+  }
 #pragma unroll
   for (int ps = 0; ps < PASSES; ++ps) {
     const int j = ps * TP + tsub;
     if ((mask >> j) & 1ull) {
-      const size_t off = head_off + (size_t)slot_token(p, a, j) * D + cidx * 8;
-      const uint4 xq = *reinterpret_cast<const uint4 *>(q + off);
-      const uint4 xk = *reinterpret_cast<const uint4 *>(k + off);
-      const uint4 xv = *reinterpret_cast<const uint4 *>(v + off);
-      const uint32_t wq[4] = {xq.x, xq.y, xq.z, xq.w}, wk[4] = {xk.x, xk.y, xk.z, xk.w},
-                     wv[4] = {xv.x, xv.y, xv.z, xv.w};
+      const uint32_t wq[4] = {xq[ps].x, xq[ps].y, xq[ps].z, xq[ps].w}, wk[4] = {xk[ps].x, xk[ps].y, xk[ps].z, xk[ps].w},
+                     wv[4] = {xv[ps].x, xv[ps].y, xv[ps].z, xv[ps].w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float f0 = bf16lo(wq[i]), f1 = bf16hi(wq[i]);
