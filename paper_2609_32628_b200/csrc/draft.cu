@@ -6,10 +6,10 @@
 // score error, so the contraction accumulates in fp64 (products of fp32 descriptors are exact there) and only the
 // final logit is rounded to fp32; with large logits (outlier channels) fp32 accumulation alone would already move
 // scores by 1e-4.  It is a small GEMM: 4*R*R*d flops per head, against 4*64*64*d flops per retained block pair in
-// the attention kernel, so the fp64 rate is not a concern.
-// 128 x 64 output tile per CTA, 8 x 4 register tile per thread, K panel of 16 channels in shared memory.  The
-// descriptors are widened to fp64 once, when a panel is staged (a conversion per use would cost more than the
-// multiply-add it feeds), and every output sums its channels in ascending order whatever the tiling.
+// the attention kernel.
+// The plain fp64 pipe sustains about half of what the fp64 tensor-core path does on this part, so the products run as
+// mma.sync m8n8k4 (fp64 in, fp64 accumulate): 128 x 64 output tile per CTA, 32 x 32 per warp (4 x 4 fragments), K
+// panels of 16 channels in shared memory.  The descriptors are widened to fp64 once, when a panel is staged.
 #include "da2_internal.cuh"
 
 namespace da2 {
@@ -17,6 +17,13 @@ namespace da2 {
 namespace {
 
 constexpr int TM = 128, TN = 64, TK = 16;
+constexpr int LDA = TM + 4, LDB = TN + 4;  // row strides = 4 mod 16 doubles: the 16 lanes of a half warp hit 16 bank pairs
+
+__device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(c[0]), "+d"(c[1])
+               : "d"(a), "d"(b));
+}
 
 __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
   const int which = blockIdx.z & 1, bh = blockIdx.z >> 1;
@@ -24,15 +31,16 @@ __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
   const float *__restrict__ Kd = p.desc[2 + which] + (size_t)bh * p.R * p.d;   // Kavg or Kmax
   float *__restrict__ out = p.logits[which] + (size_t)bh * p.R * p.R;
   const int a0 = blockIdx.y * TM, b0 = blockIdx.x * TN;
-  __shared__ __align__(16) double As[TK][TM + 2];
-  __shared__ __align__(16) double Bs[TK][TN + 2];
-  const int tid = threadIdx.x;
-  const int tx = tid & 15, ty = tid >> 4;  // thread tile: rows ty*8.., cols tx*4..
-  double acc[8][4];
+  __shared__ __align__(16) double As[TK][LDA];  // [channel][query block]
+  __shared__ __align__(16) double Bs[TK][LDB];  // [channel][key block]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 3) * 32, wn = (warp >> 2) * 32;  // warp tile origin inside the CTA tile
+  const int fr = lane >> 2, fc = lane & 3;                // fragment row (or column of B) and channel inside a k4 step
+  double acc[4][4][2];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int j = 0; j < 4; ++j) { acc[i][j][0] = 0.0; acc[i][j][1] = 0.0; }
 
   // loader mapping: 64 rows x 16 channels = 256 float4 quarters -> one float4 per thread per 64 rows
   const int lr = tid >> 2, lc = (tid & 3) * 4;
@@ -47,32 +55,28 @@ __global__ void __launch_bounds__(256) draft_logits_kernel(Params p) {
     Bs[lc + 0][lr] = xb.x; Bs[lc + 1][lr] = xb.y; Bs[lc + 2][lr] = xb.z; Bs[lc + 3][lr] = xb.w;
     __syncthreads();
 #pragma unroll
-    for (int kk = 0; kk < TK; ++kk) {
-      double ar[8], br[4];
+    for (int k4 = 0; k4 < TK; k4 += 4) {
+      double af[4], bf[4];
 #pragma unroll
-      for (int i = 0; i < 8; i += 2) {
-        const double2 t = *reinterpret_cast<const double2 *>(&As[kk][ty * 8 + i]);
-        ar[i] = t.x; ar[i + 1] = t.y;
-      }
+      for (int i = 0; i < 4; ++i) af[i] = As[k4 + fc][wm + i * 8 + fr];
 #pragma unroll
-      for (int j = 0; j < 4; j += 2) {
-        const double2 t = *reinterpret_cast<const double2 *>(&Bs[kk][tx * 4 + j]);
-        br[j] = t.x; br[j + 1] = t.y;
-      }
+      for (int j = 0; j < 4; ++j) bf[j] = Bs[k4 + fc][wn + j * 8 + fr];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fma(ar[i], br[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) dmma(acc[i][j], af[i], bf[j]);
     }
   }
+  // accumulator fragment: row = lane / 4, columns 2 * (lane % 4) and + 1
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int a = a0 + ty * 8 + i;
+  for (int i = 0; i < 4; ++i) {
+    const int a = a0 + wm + i * 8 + fr;
     if (a >= p.R) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int b = b0 + tx * 4 + j;
-      if (b < p.R) out[(size_t)a * p.R + b] = (float)((double)p.scale * acc[i][j]);
+      const int b = b0 + wn + j * 8 + fc * 2;
+      if (b < p.R) out[(size_t)a * p.R + b] = (float)((double)p.scale * acc[i][j][0]);
+      if (b + 1 < p.R) out[(size_t)a * p.R + b + 1] = (float)((double)p.scale * acc[i][j][1]);
     }
   }
 }
