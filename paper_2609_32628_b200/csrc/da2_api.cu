@@ -3,6 +3,9 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <map>
+#include <mutex>
+#include <tuple>
 #include <vector>
 
 #include "da2_internal.cuh"
@@ -131,6 +134,23 @@ BandChoice choose_bands(int H, int W, int Rf) {
   return best;
 }
 
+// The search costs a few milliseconds and depends on the frame's grid only: plans of the same grid (the per-group plans
+// of the host entry, for one) share its result.
+BandChoice cached_bands(int H, int W, int Rf) {
+  static std::mutex mu;
+  static std::map<std::tuple<int, int, int>, BandChoice> memo;
+  const auto key = std::make_tuple(H, W, Rf);
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find(key);
+    if (it != memo.end()) return it->second;
+  }
+  const BandChoice ch = choose_bands(H, W, Rf);
+  std::lock_guard<std::mutex> lock(mu);
+  memo.emplace(key, ch);
+  return ch;
+}
+
 // kernels enqueued by the calling thread's last da2_prepare / da2_refresh_operands / da2_attention_fwd
 thread_local int t_last_launches = 0;
 
@@ -181,7 +201,7 @@ da2_status_t da2_plan(const da2_config_t *cfg, da2_plan_t **plan_out) {
   if (cfg->partition == DA2_PARTITION_BALANCED) {
     const int HW = cfg->Hg * cfg->Wg;
     I.R_f = (HW + da2::kSlots - 1) / da2::kSlots;
-    const BandChoice ch = choose_bands(cfg->Hg, cfg->Wg, I.R_f);
+    const BandChoice ch = cached_bands(cfg->Hg, cfg->Wg, I.R_f);
     I.part_transposed = ch.transposed;
     I.part_bands = ch.bands;
     I.part_perimeter = ch.perimeter;
