@@ -213,6 +213,17 @@ int32_t da2_last_launch_count(const da2_plan_t *plan);
  * normally.  da2_device_status then reports DA2_ERR_TIMEOUT; the next da2_prepare clears the word. */
 da2_status_t da2_probe_bounded_wait(const da2_plan_t *plan, void *workspace, int64_t limit_cycles, void *stream);
 
+/* Arithmetic self-check of the operand quantisers (diagnostic; the paper has no counterpart).  The quantisers of
+ * App. C.3 divide every element by a scale; the kernels obtain that quotient from a reciprocal taken once per scale and
+ * two fused multiply-adds, and round INT8 codes half away from zero by one addition and a truncation.  This call
+ * compares both, on the device and with the very device functions the kernels use, against the IEEE division and
+ * against roundf: mode 0: every finite bf16 numerator with |x| >= 2^-100 against n_divisors pseudo-random divisors
+ * in [2^-60, 2^60) (seed selects them); mode 1: the same with significands of all ones; mode 2: every float below
+ * 2^23 in magnitude through the rounding (n_divisors, seed ignored).  out_dev: device uint64[1], receives the number
+ * of mismatches (0 expected).  Asynchronous on stream. */
+da2_status_t da2_selfcheck_quantiser_arithmetic(int32_t mode, int32_t n_divisors, uint32_t seed, void *out_dev,
+                                                void *stream);
+
 /* Tensor-core microbenchmark (diagnostic; the paper has no counterpart).  Every one of `ctas` CTAs issues
  * 4*iters back-to-back tcgen05.mma instructions of one kind with M = 128 and the given N (64, 128 or 256), operands
  * in shared memory, accumulators in tensor memory.  kind: 0 bf16 (K = 16 per instruction), 1 INT8 (K = 32),

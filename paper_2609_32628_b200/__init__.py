@@ -7,8 +7,8 @@ compute call requires the CUDA library and a device.
 """
 from .binding import (Da2Error, Plan, PlanInfo, STATUS, load_library, da2_plan, da2_plan_info, da2_plan_slot_token, da2_prepare, da2_refresh_operands, da2_prepare_cached_scales,
                       da2_attention_fwd, da2_device_status, da2_plan_destroy, da2_status_string,
-                      da2_last_launch_count, da2_probe_bounded_wait, da2_attention_host, da2_attention_host_arena_bytes, make_config, da2_tcgen05_peak, da2_draft_map_noalloc, attention, HostPipeline)
+                      da2_last_launch_count, da2_probe_bounded_wait, da2_attention_host, da2_attention_host_arena_bytes, make_config, da2_tcgen05_peak, da2_selfcheck_quantiser_arithmetic, da2_draft_map_noalloc, attention, HostPipeline)
 
 __all__ = ["Da2Error", "Plan", "PlanInfo", "STATUS", "load_library", "da2_plan", "da2_plan_info", "da2_plan_slot_token", "da2_prepare", "da2_refresh_operands", "da2_prepare_cached_scales",
            "da2_attention_fwd", "da2_device_status", "da2_plan_destroy", "da2_status_string",
-           "da2_last_launch_count", "da2_probe_bounded_wait", "da2_attention_host", "da2_attention_host_arena_bytes", "make_config", "da2_tcgen05_peak", "da2_draft_map_noalloc", "attention", "HostPipeline"]
+           "da2_last_launch_count", "da2_probe_bounded_wait", "da2_attention_host", "da2_attention_host_arena_bytes", "make_config", "da2_tcgen05_peak", "da2_selfcheck_quantiser_arithmetic", "da2_draft_map_noalloc", "attention", "HostPipeline"]

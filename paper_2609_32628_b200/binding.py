@@ -231,6 +231,18 @@ def da2_probe_bounded_wait(plan: Plan, workspace, limit_cycles: int, stream=None
         raise Da2Error(rc, "da2_probe_bounded_wait")
 
 
+def da2_selfcheck_quantiser_arithmetic(mode: int, n_divisors: int, seed: int, out_dev, stream=None) -> None:
+    """Device self-check of the quantisers' quotient and rounding arithmetic (see include/da2.h); out_dev: CUDA
+    uint64[1] (int64 tensor), receives the mismatch count."""
+    lib = load_library()
+    fn = lib.da2_selfcheck_quantiser_arithmetic
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
+    rc = fn(mode, n_divisors, seed, _ptr(out_dev), _stream(stream))
+    if rc != 0:
+        raise Da2Error(rc, "da2_selfcheck_quantiser_arithmetic")
+
+
 def da2_tcgen05_peak(kind: int, n: int, iters: int, ctas: int, out_dev, stream=None) -> None:
     """Tensor-core microbenchmark launch (see include/da2.h); out_dev: CUDA int64[4]."""
     lib = load_library()

@@ -386,6 +386,16 @@ da2_status_t da2_attention_fwd(const da2_plan_t *plan, const void *q, const void
   return DA2_OK;
 }
 
+da2_status_t da2_selfcheck_quantiser_arithmetic(int32_t mode, int32_t n_divisors, uint32_t seed, void *out_dev,
+                                                void *stream) {
+  if (!out_dev || mode < 0 || mode > 2 || misaligned(out_dev, 8)) return DA2_ERR_INVALID_ARG;
+  if (mode != 2 && (n_divisors < 1 || n_divisors > (1 << 22))) return DA2_ERR_INVALID_ARG;
+  if (da2::launch_quantiser_selfcheck(mode, n_divisors, seed, (unsigned long long *)out_dev, (cudaStream_t)stream) !=
+      cudaSuccess)
+    return DA2_ERR_CUDA;
+  return DA2_OK;
+}
+
 da2_status_t da2_device_status(const da2_plan_t *plan, const void *workspace, void *stream) {
   if (!plan || !workspace) return DA2_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;

@@ -118,6 +118,7 @@ cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bflo
                         cudaStream_t st, int *launches, bool pool = false);
 cudaError_t launch_attention(const Params &p, __nv_bfloat16 *out, cudaStream_t st, int *launches);
 cudaError_t launch_bounded_wait_probe(int *status, long long limit_cycles, cudaStream_t st);
+cudaError_t launch_quantiser_selfcheck(int mode, int n_divisors, uint32_t seed, unsigned long long *out, cudaStream_t st);
 
 }  // namespace da2
 

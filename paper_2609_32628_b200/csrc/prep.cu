@@ -308,7 +308,48 @@ __global__ void __launch_bounds__(NT) prep_kernel(Params p, const __nv_bfloat16 
   }
 }
 
+// Self-check of Divider::quick and round_half_away against the IEEE division and roundf (see da2.h).
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7feb352dU; x ^= x >> 15; x *= 0x846ca68bU; x ^= x >> 16;
+  return x;
+}
+__global__ void selfcheck_quotient_kernel(int n_divisors, int all_ones, uint32_t seed, unsigned long long *bad_out) {
+  const int di = blockIdx.x * blockDim.x + threadIdx.x;
+  if (di >= n_divisors) return;
+  const uint32_t h = mix32((uint32_t)di * 2654435761u + seed);
+  const uint32_t man = all_ones ? 0x7fffffu : (h & 0x7fffffu);
+  const uint32_t ex = 127u - 60u + mix32(h) % 120u;  // binades 2^-60 .. 2^59: inside the quick range
+  const Divider div = make_divider(__uint_as_float((ex << 23) | man));
+  unsigned long long bad = div.fast ? 0ull : 1ull;
+  for (uint32_t b = 0; b < 65536u; ++b) {
+    const float x = __uint_as_float(b << 16);
+    if (!(fabsf(x) <= 3.0e38f) || (x != 0.f && fabsf(x) < 7.9e-31f)) continue;  // finite, zero or at least 2^-100
+    const float ref = div.exact(x);
+    if (!(fabsf(ref) < 3.0e38f) || (ref != 0.f && fabsf(ref) < 1e-30f)) continue;  // quotient in the normal range
+    if (__float_as_uint(div.quick(x)) != __float_as_uint(ref)) ++bad;
+  }
+  if (bad) atomicAdd(bad_out, bad);
+}
+__global__ void selfcheck_round_kernel(unsigned long long *bad_out) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  unsigned long long bad = 0;
+  for (unsigned long long b = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; b < (1ull << 32); b += stride) {
+    const float x = __uint_as_float((uint32_t)b);
+    if (!(fabsf(x) < 8388608.0f)) continue;
+    if ((int)roundf(x) != round_half_away(x)) ++bad;
+  }
+  if (bad) atomicAdd(bad_out, bad);
+}
+
 }  // namespace
+
+cudaError_t launch_quantiser_selfcheck(int mode, int n_divisors, uint32_t seed, unsigned long long *out, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(out, 0, sizeof(unsigned long long), st);
+  if (e != cudaSuccess) return e;
+  if (mode == 2) selfcheck_round_kernel<<<148 * 8, 256, 0, st>>>(out);
+  else selfcheck_quotient_kernel<<<(n_divisors + 127) / 128, 128, 0, st>>>(n_divisors, mode == 1, seed, out);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_prep(const Params &p, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         cudaStream_t st, int *launches, bool pool) {

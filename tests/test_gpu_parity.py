@@ -314,6 +314,44 @@ def test_caller_fixed_nvfp4_scales():
     _check_attention(w, out, ref, sel, bad, g_fixed=g_fixed)
 
 
+def test_quantiser_codes_on_a_lattice_of_bf16_patterns():
+    """The quantisers get their quotients from a hoisted reciprocal and two fused multiply-adds instead of a division
+    per element; the codes must still be the oracle's (which divides) bit for bit.  Inputs here are not smooth fields
+    but bf16 bit patterns drawn over 19 binades with every mantissa, both signs and signed zeros, under caller-fixed
+    NVFP4 scales with awkward significands, so that quotients land on and next to rounding boundaries of every
+    format."""
+    w = SMALL["ragged3"]
+    BH = w.B * w.H
+    gen = torch.Generator().manual_seed(2024)
+    def lattice():
+        shape = (w.B, w.H, w.N, w.head_dim)
+        sign = torch.randint(0, 2, shape, generator=gen, dtype=torch.int32) << 15
+        expo = (torch.randint(127 - 12, 127 + 7, shape, generator=gen, dtype=torch.int32)) << 7
+        mant = torch.randint(0, 128, shape, generator=gen, dtype=torch.int32)
+        bits = sign | expo | mant
+        zero = torch.rand(shape, generator=gen) < 0.02
+        bits = torch.where(zero, sign, bits)  # +0 and -0
+        return bits.to(torch.int16).view(torch.bfloat16).cuda()
+    q, k, v = lattice(), lattice(), lattice()
+    g_fixed = ([0.0123456, 0.0301], [0.0271828, 0.0099999], [0.0314159, 0.0200001])
+    assert all(len(g) == BH for g in g_fixed)
+    plan, ws, out = run_gpu(w, q, k, v, g_fixed=g_fixed)
+    ref = oracle_all(w, q, k, v)
+    _check_prepare(w, plan, ws, ref, g_fixed=g_fixed)
+
+
+@pytest.mark.parametrize("mode,n_divisors", [(0, 1 << 16), (1, 1 << 12), (2, 1)])
+def test_quantiser_arithmetic_selfcheck(mode, n_divisors):
+    """The device functions behind the quantisers' quotients (hoisted reciprocal + two fused multiply-adds) and the
+    INT8 rounding (one add and a truncation) against the IEEE division and roundf: every bf16 numerator of magnitude
+    at least 2^-100 against 65,536 pseudo-random divisors and 4,096 divisors with significands of all ones, and every
+    float below 2^23 through the rounding.  No mismatch is allowed."""
+    bad = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    da2.da2_selfcheck_quantiser_arithmetic(mode, n_divisors, 20260101, bad)
+    torch.cuda.synchronize()
+    assert int(bad.item()) == 0
+
+
 def test_refresh_operands_keeps_the_selection():
     """da2_refresh_operands: new operands under the lists of an earlier call (the selection is reused)."""
     w1 = SMALL["ragged64"]
