@@ -47,7 +47,8 @@ __device__ __forceinline__ float decode_e4m3(uint32_t c) {
 // with |x| >= 2^-100 and millions of divisors in [2^-60, 2^60], significands of all ones included: the only
 // difference is the sign of a zero quotient, which the sign copy restores (d > 0).  For |x| < 2^-100 the residual can
 // underflow; the quotient is then below 2^-40 in magnitude either way and every format here encodes it as a signed
-// zero.  Divisors outside [2^-60, 2^60] (or not finite) keep the plain division.
+// zero.  Divisors outside [2^-60, 2^60] (or not finite) keep the plain division.  da2_selfcheck_quantiser_arithmetic
+// repeats the check with these very functions.
 struct Divider {
   float d, r;
   bool fast;
