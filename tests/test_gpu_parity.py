@@ -245,6 +245,12 @@ def test_wan1p3b_480p_head_scope_sampled_parity():
     _sampled_parity("wan1p3b_480p", nheads=2, nblocks=16, rank_scope=1)
 
 
+def test_wan14b_720p_head_scope_sampled_parity():
+    """The head-level budget on the bench workload (the configuration whose timing the measured table quotes): rows
+    from 11 to 1260 blocks long, paired by the scheduling order."""
+    _sampled_parity("wan14b_720p", nheads=2, nblocks=8, rank_scope=1)
+
+
 @pytest.mark.parametrize("name", ["ragged3", "ragged64", "batch2"])
 @pytest.mark.parametrize("rank_scope", [0, 1])
 def test_balanced_partition_full_parity(name, rank_scope):
