@@ -298,7 +298,7 @@ def attention(plan: Plan, q, k, v, workspace=None, out=None, stream=None):
 class HostPipeline:
     """Attention on HOST tensors with the PCIe copies hidden behind the kernels.
 
-    Heads are independent problems, so the call is cut into groups of heads that flow through three CUDA streams:
+    Heads are independent problems, so the call is cut into groups of heads that flow through four CUDA streams:
     host-to-device copies of group g+1, da2_prepare + da2_attention_fwd of group g and the device-to-host copy of
     group g-1 run at the same time (two device slots per stage).  Everything that computes is the same C ABI; this
     class only owns the per-group plans, buffers, streams and events.  Inputs and output must be pinned host tensors
@@ -326,7 +326,10 @@ class HostPipeline:
                            ws=torch.empty(wsb, dtype=torch.uint8, device=self.device)) for _ in range(2)]
         for slot in self.slots:
             slot["ws"][:256].zero_()   # status words read as OK until a call writes them
-        self.s_in, self.s_c, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
+        self.s_in, self.s_out = (torch.cuda.Stream(self.device) for _ in range(2))
+        # one compute stream per device slot: consecutive groups share nothing, so the first kernels of group g+1 fill
+        # the SMs that the last, partly filled wave of group g's attention kernel leaves idle
+        self.s_cs = [torch.cuda.Stream(self.device) for _ in range(2)]
         self.launches = 0
         # one status word per head group, copied out after the group's kernels: the next group that reuses the slot
         # clears the slot's word, so the slots alone would only remember the last two groups
@@ -357,13 +360,13 @@ class HostPipeline:
         current stream waits for the last copy."""
         torch = self.torch
         cur = torch.cuda.current_stream(self.device)
-        for s in (self.s_in, self.s_c, self.s_out):
+        for s in (self.s_in, self.s_out, *self.s_cs):
             s.wait_stream(cur)
         fq, fk, fv, fo = (t.view(self.BH, self.N, self.d) for t in (hq, hk, hv, hout))
         ev_c, ev_out = [], []
         self.launches = 0
         for gi, (a, b) in enumerate(self.ranges):
-            n, slot = b - a, self.slots[gi % 2]
+            n, slot, s_c = b - a, self.slots[gi % 2], self.s_cs[gi % 2]
             plan = self.plans[n]
             q, k, v, o = (slot[x][:n] for x in ("q", "k", "v", "out"))
             with torch.cuda.stream(self.s_in):
@@ -374,19 +377,19 @@ class HostPipeline:
                 v.copy_(fv[a:b], non_blocking=True)
                 e_in = torch.cuda.Event()
                 e_in.record(self.s_in)
-            with torch.cuda.stream(self.s_c):
-                self.s_c.wait_event(e_in)
+            with torch.cuda.stream(s_c):
+                s_c.wait_event(e_in)
                 if gi >= 2:
-                    self.s_c.wait_event(ev_out[gi - 2])      # the slot's previous output has left the device
+                    s_c.wait_event(ev_out[gi - 2])           # the slot's previous output has left the device
                 q4, k4, v4, o4 = (t.view(1, n, self.N, self.d) for t in (q, k, v, o))
-                da2_prepare(plan, q4, k4, v4, slot["ws"], self.s_c)
+                da2_prepare(plan, q4, k4, v4, slot["ws"], s_c)
                 self.launches += da2_last_launch_count(plan)
-                da2_attention_fwd(plan, q4, k4, v4, slot["ws"], o4, self.s_c)
+                da2_attention_fwd(plan, q4, k4, v4, slot["ws"], o4, s_c)
                 self.launches += da2_last_launch_count(plan)
                 off = int(plan.info.off_status)
                 self.group_status[gi].copy_(slot["ws"][off:off + 16].view(torch.int32), non_blocking=True)
                 e_c = torch.cuda.Event()
-                e_c.record(self.s_c)
+                e_c.record(s_c)
                 ev_c.append(e_c)
             with torch.cuda.stream(self.s_out):
                 self.s_out.wait_event(e_c)
@@ -395,7 +398,8 @@ class HostPipeline:
                 e_o.record(self.s_out)
                 ev_out.append(e_o)
         cur.wait_stream(self.s_out)
-        cur.wait_stream(self.s_c)
+        for s in self.s_cs:
+            cur.wait_stream(s)
 
     def status(self) -> int:
         """Worst device status over all head groups of the last run (synchronises): 0 = DA2_OK, 5 = DA2_ERR_TIMEOUT

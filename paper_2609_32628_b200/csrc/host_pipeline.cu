@@ -1,7 +1,7 @@
 // da2_attention_host: the whole call on HOST tensors with the PCIe copies hidden behind the kernels.
 //
 // Heads are independent problems (pooling, ranking, preparation and attention never mix heads), so the call is cut
-// into groups of heads that flow through three streams: the host-to-device copy of group g+1, da2_prepare +
+// into groups of heads that flow through four streams: the host-to-device copy of group g+1, da2_prepare +
 // da2_attention_fwd of group g and the device-to-host copy of group g-1 run at the same time, on two device slots
 // carved out of one caller-provided arena.  Groups are small at both ends (the first copy-in and the last copy-out
 // are the only transfers that nothing hides) and large in between.  Everything that computes is the C ABI above.
@@ -98,11 +98,14 @@ da2_status_t da2_attention_host(const da2_config_t *cfg, const void *hq, const v
   const da2_plan_info_t &I0 = plans.begin()->second->info;
   const size_t head_bytes = (size_t)(I0.N + I0.n_prefix) * I0.head_dim * 2;
   const int G = (int)L.groups.size();
-  cudaStream_t s_in = nullptr, s_c = nullptr, s_out = nullptr;
+  // one compute stream per device slot: consecutive groups share nothing, so the first kernels of group g+1 fill the
+  // SMs that the last, partly filled wave of group g's attention kernel leaves idle
+  cudaStream_t s_in = nullptr, s_cs[2] = {nullptr, nullptr}, s_out = nullptr;
   std::vector<cudaEvent_t> e_in(G, nullptr), e_c(G, nullptr), e_out(G, nullptr);
   std::vector<int> status(4 * (size_t)G, 0);
   bool ok = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
-            cudaStreamCreateWithFlags(&s_c, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&s_cs[0], cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&s_cs[1], cudaStreamNonBlocking) == cudaSuccess &&
             cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
   for (int g = 0; ok && g < G; ++g)
     ok = cudaEventCreateWithFlags(&e_in[g], cudaEventDisableTiming) == cudaSuccess &&
@@ -118,6 +121,7 @@ da2_status_t da2_attention_host(const da2_config_t *cfg, const void *hq, const v
     uint8_t *ws = slot + 4 * L.tensor_bytes;
     const size_t off = (size_t)first * head_bytes, bytes = (size_t)n * head_bytes;
     da2_plan_t *plan = plans[n];
+    cudaStream_t s_c = s_cs[g & 1];
     ok = true;
     if (g >= 2) ok = cudaStreamWaitEvent(s_in, e_c[g - 2], 0) == cudaSuccess;  // the slot's inputs were consumed
     ok = ok && cudaMemcpyAsync(dq, (const uint8_t *)hq + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
@@ -139,7 +143,7 @@ da2_status_t da2_attention_host(const da2_config_t *cfg, const void *hq, const v
     first += n;
   }
   // the call is synchronous: everything enqueued above has finished when it returns
-  for (cudaStream_t s : {s_in, s_c, s_out})
+  for (cudaStream_t s : {s_in, s_cs[0], s_cs[1], s_out})
     if (s && cudaStreamSynchronize(s) != cudaSuccess && st == DA2_OK) st = DA2_ERR_CUDA;
   if (st == DA2_OK && cudaMemcpy(status.data(), dev_status, 16 * (size_t)G, cudaMemcpyDeviceToHost) != cudaSuccess)
     st = DA2_ERR_CUDA;
@@ -154,7 +158,7 @@ da2_status_t da2_attention_host(const da2_config_t *cfg, const void *hq, const v
     if (e_c[g]) cudaEventDestroy(e_c[g]);
     if (e_out[g]) cudaEventDestroy(e_out[g]);
   }
-  for (cudaStream_t s : {s_in, s_c, s_out})
+  for (cudaStream_t s : {s_in, s_cs[0], s_cs[1], s_out})
     if (s) cudaStreamDestroy(s);
   destroy_plans(plans);
   return st;
