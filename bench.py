@@ -390,7 +390,7 @@ def run_da2(args, rank, world, local_rank):
                    "l2": "inputs larger than L2 (Q, K, V and operand records are several GB per step)"},
         "e2e": {"value": dense * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": out.numel() * 2,
-                "how": f"HostPipeline: groups of {groups} heads, copy-in / kernels / copy-out on three streams, "
+                "how": f"HostPipeline: groups of {groups} heads, copy-in, copy-out and two alternating compute streams, "
                        f"{e2e_launches} kernels per step",
                 "c_abi_host_entry_ms_per_step": e2e_c_ms,
                 "serial_ms_per_step": e2e_serial_ms,
