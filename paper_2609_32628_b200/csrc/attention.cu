@@ -834,24 +834,39 @@ __global__ void __launch_bounds__(Roles<SETS>::NT, 1) attention_kernel(Params p,
         continue;
       }
       const int tier = S.tier(i);
-      if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & kMask)), ((i - 1) >> kShift) & 1, abortp)) break;
-      tc::fence_after_sync();
+      // everything that does not need the accumulator comes before the wait for product i-1
       float lane_factor = 1.0f;
       if (tier_switch && ch < D) {
         const float un = unit_of(tier), up = unit_of(S.tier(i - 1));
         lane_factor = un > 0.f ? __fdiv_rn(up, un) : 0.f;
       }
       const float *fac = s_factor + (s * kSets + g) * 64;
+      // column groups (eight queries each) with a moved maximum; all of them when the segment changes.  Two groups
+      // are in flight at a time: their loads are issued together, so a rescale costs one TMEM round trip per pair.
+      uint32_t todo = 0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        if (tier_switch || (((c < 4 ? moved.x : moved.y) >> ((c & 3) * 8)) & 0xffu) != 0u) todo |= 1u << c;
+      if (!wait_or_abort(bar(s, B_PVDONE + ((i - 1) & kMask)), ((i - 1) >> kShift) & 1, abortp)) break;
+      tc::fence_after_sync();
 #pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        const uint32_t m8 = ((c < 4 ? moved.x : moved.y) >> ((c & 3) * 8)) & 0xffu;
-        if (m8 == 0u && !tier_switch) continue;
-        uint32_t o[8];
-        tc::tmem_ld8(tmem + lane_addr + col_o(s) + c * 8, o);
+      while (todo) {
+        const int c0 = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int c1 = todo ? __ffs(todo) - 1 : -1;
+        if (c1 >= 0) todo &= todo - 1;
+        uint32_t o0[8], o1[8];
+        tc::tmem_ld8(tmem + lane_addr + col_o(s) + c0 * 8, o0);
+        if (c1 >= 0) tc::tmem_ld8(tmem + lane_addr + col_o(s) + c1 * 8, o1);
         tc::wait_ld();
 #pragma unroll
-        for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * (fac[c * 8 + j] * lane_factor));
-        tc::tmem_st8(tmem + lane_addr + col_o(s) + c * 8, o);
+        for (int j = 0; j < 8; ++j) o0[j] = __float_as_uint(__uint_as_float(o0[j]) * (fac[c0 * 8 + j] * lane_factor));
+        tc::tmem_st8(tmem + lane_addr + col_o(s) + c0 * 8, o0);
+        if (c1 >= 0) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) o1[j] = __float_as_uint(__uint_as_float(o1[j]) * (fac[c1 * 8 + j] * lane_factor));
+          tc::tmem_st8(tmem + lane_addr + col_o(s) + c1 * 8, o1);
+        }
       }
       tc::wait_st();
       tc::fence_before_sync();
